@@ -1,0 +1,186 @@
+/* wpsgd.h -- C ABI of the B200 (sm_100a) library for the hot path of weighted parallel SGD.
+ *
+ * Method: Cheng, Li, Zhang, "Weighted parallel SGD for distributed unbalanced-workload
+ * training system" (WP-SGD). The library runs Algorithm 1 on one GPU:
+ *
+ *   - k simulated nodes; node j owns the rows [shard_off[j], shard_off[j+1]) of the data and
+ *     runs n_steps[j] sequential SGD steps (Eq. 5) on the regularised loss of Eq. 4,
+ *         w_n = w_{n-1} - eta_n ( lambda w_{n-1} + L'(y, w_{n-1}.x) x ),
+ *     starting from a shared w0 (zeros if not given). Chains of different nodes are independent.
+ *   - the final models are combined with the weights of Eq. 6 (default rate r = 1 - eta lambda)
+ *     or Eq. 8 (caller's rate r):  v = sum_j weight_j w_j,  weight_j = r^{T_j} / sum_i r^{T_i},
+ *     where T_j = max_i n_steps[i] - n_steps[j] is the paper's delay of node j.
+ *
+ * Conventions fixed here because the paper leaves them open:
+ *   - The n-th example (n = 1, 2, ...) of node j is row shard_off[j] + floor(u m_j / 2^32), where
+ *     m_j is the shard's row count and u is output word (n-1) mod 4 of Philox4x32-10 with key
+ *     (seed low 32 bits, seed high 32 bits) and counter ((n-1)/4 low, (n-1)/4 high, j, 0):
+ *     i.i.d. uniform draws with replacement, a pure function of (seed, j, n).
+ *   - Losses, with z = w.x: hinge L = max(0, 1 - y z), L' = -y if y z < 1 else 0;
+ *     logistic L = log(1 + exp(-y z)), L' = -y / (1 + exp(y z)); squared L = (z - y)^2 / 2,
+ *     L' = z - y. Labels for hinge and logistic are +1 / -1 floats.
+ *   - Step size: constant eta0, or eta_n = eta0 / sqrt(n). For the decaying schedule the default
+ *     weight of node j is the product of (1 - eta_s lambda) over the steps s = n_j+1 .. t it did
+ *     not run (this equals Eq. 6 when eta is constant; the paper has constant eta only).
+ *   - A node with n_steps[j] == 0 keeps w0 and still takes part in the combination.
+ *
+ * Arithmetic: features fp32 or bf16 (widened exactly), model and accumulation fp32, the scale
+ * factor of the sparse path and all weights fp64.
+ *
+ * Memory: every pointer is tagged DEVICE or HOST below. Device buffers belong to the caller and
+ * must stay valid until the work enqueued on the context's stream has finished. The context owns
+ * the k x d model matrix, the index stream and small tables. All functions except the *_host one
+ * and the queries documented as synchronous only enqueue work on the stream given at creation.
+ *
+ * Errors: every function returns a wpsgd_status; a text for the last failure on a context is
+ * available from wpsgd_last_error(). Nothing throws or aborts. Kernels never spin without bound:
+ * a wait that exceeds its limit sets a device status word, reported as WPSGD_ERR_TIMEOUT by the
+ * next wpsgd_check().
+ */
+#ifndef WPSGD_H_
+#define WPSGD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wpsgd_ctx wpsgd_ctx; /* opaque; created and destroyed by the library */
+
+typedef enum {
+  WPSGD_OK = 0,
+  WPSGD_ERR_INVALID_ARG = 1,
+  WPSGD_ERR_ALLOC = 2,
+  WPSGD_ERR_CUDA = 3,
+  WPSGD_ERR_STATE = 4,       /* call out of order, e.g. combine before run */
+  WPSGD_ERR_UNSUPPORTED = 5,
+  WPSGD_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up */
+} wpsgd_status;
+
+typedef enum { WPSGD_LOSS_HINGE = 0, WPSGD_LOSS_LOGISTIC = 1, WPSGD_LOSS_SQUARED = 2 } wpsgd_loss;
+typedef enum { WPSGD_X_F32 = 0, WPSGD_X_BF16 = 1 } wpsgd_xtype;
+typedef enum { WPSGD_LR_CONST = 0, WPSGD_LR_INV_SQRT = 1 } wpsgd_lr;
+
+/* Create a context for k nodes and d features on CUDA device `device`; all work is enqueued on
+ * `cuda_stream` (a cudaStream_t; NULL = the legacy default stream). Allocates the k x d fp32
+ * model matrix. (Algorithm 1: inputs "nodes k", model w in R^d.) */
+wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, wpsgd_ctx** out);
+
+/* Release everything the context owns. Synchronises the stream first. NULL is accepted. */
+wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
+
+/* Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
+ * with register-held model, 3 warp per node, 4 blocked cluster kernel), "prefetch" (rows in
+ * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "block_rows" (rows per block of the blocked kernel), "cluster" (CTAs per
+ * node of the blocked kernel), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
+ * (iterations after which a device-side wait gives up), "timing" (1: record events around the chain kernel). Unknown name or bad value:
+ * WPSGD_ERR_INVALID_ARG. The result of a run never depends on these beyond rounding order. */
+wpsgd_status wpsgd_set_option(wpsgd_ctx* ctx, const char* name, int64_t value);
+
+/* Node numbers that enter the sample stream in place of 0..k-1 (HOST [k], >= 0; NULL restores the
+ * default). A GPU that holds a subset of a larger cluster's nodes passes their global numbers, so
+ * that every node draws the same examples wherever it is placed. Takes effect at the next run. */
+wpsgd_status wpsgd_set_node_ids(wpsgd_ctx* ctx, const int32_t* ids);
+
+/* Algorithm 1, the per-node loops (Eq. 5), on dense rows.
+ *   X          DEVICE  [N, ld_elems] row-major, fp32 or bf16 per `xt`; only the first d columns
+ *                      of a row are read. N = shard_off[k].
+ *   y          DEVICE  [N] fp32 labels / targets.
+ *   shard_off  HOST    [k+1] non-decreasing row offsets; node j owns rows [off[j], off[j+1]).
+ *   n_steps    HOST    [k] steps of each node (>= 0). A node with steps needs >= 1 row, < 2^32 rows.
+ *   eta0, sched, lambda, loss   as in the header comment; requires 0 <= eta_n lambda < 1.
+ *   seed       seed of the sample stream.
+ *   w0         DEVICE  [d] shared initial model, or NULL for zeros (Algorithm 1 initialises to 0;
+ *                      the paper's experiments start from a constant vector).
+ * After the call the context holds the k final models. Host arrays are copied before return. */
+wpsgd_status wpsgd_run(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                       const int64_t* shard_off, const int64_t* n_steps, float eta0, wpsgd_lr sched,
+                       float lambda, wpsgd_loss loss, uint64_t seed, const float* w0);
+
+/* Continue every chain from the models the context holds: node j runs n_more[j] further steps,
+ * numbered after the ones it has already run (so it draws examples step_done+1, ...). Data and
+ * hyper-parameters must be the ones given to the wpsgd_run / wpsgd_run_csr that started the
+ * chains. Gives the paper's snapshots "after 100000 x i updates of the fastest node"
+ * (Section "Numerical experiments", Approach) without restarting. Dense data only. */
+wpsgd_status wpsgd_continue(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                            const int64_t* shard_off, const int64_t* n_more);
+
+/* The same loops on sparse rows in CSR form (the paper's data: a few tens of features per row).
+ *   row_ptr    DEVICE  [N+1] int64, col_idx DEVICE [nnz] int32 (unique within a row, < d),
+ *   val        DEVICE  [nnz] fp32.  Other arguments as wpsgd_run.
+ * The model of node j is kept as s_j * u_j with an fp64 scalar s_j, so that the regulariser costs
+ * one scalar multiply per step instead of a pass over d (same iterates as Eq. 5). */
+wpsgd_status wpsgd_run_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                           const float* y, const int64_t* shard_off, const int64_t* n_steps, float eta0,
+                           wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed, const float* w0);
+
+/* Algorithm 1, the aggregation: v = sum_j weight_j w_j (j ascending) with Eq. 6 weights, or Eq. 8
+ * weights when r > 0 is given (r <= 0 or NaN selects the default; r = 1 is plain averaging).
+ *   v_out      DEVICE  [d] fp32.
+ * WPSGD_ERR_STATE if no run has been made on the context. */
+wpsgd_status wpsgd_combine(wpsgd_ctx* ctx, double r, float* v_out);
+
+/* The same aggregation with weights given by the caller (HOST [k] fp64): v = sum_j weights[j] w_j.
+ * For a cluster of GPUs that each hold a subset of the nodes: every GPU passes the Eq. 6 weights of
+ * its own nodes, computed over all nodes with wpsgd_weights, and the partial sums are then added
+ * across GPUs (the single exchange of Algorithm 1's last line). */
+wpsgd_status wpsgd_combine_weighted(wpsgd_ctx* ctx, const double* weights, float* v_out);
+
+/* Copy the k final models (W^{j, t - T_j} of Lemma 3), scale applied, to W_out DEVICE [k, d] fp32. */
+wpsgd_status wpsgd_get_models(wpsgd_ctx* ctx, float* W_out);
+
+/* Replace every node's model by v (DEVICE [d]): the broadcast step of averaging every `span`
+ * fastest-node steps (Section "Combining WP-SGD with bucket SGD"); follow with wpsgd_continue. */
+wpsgd_status wpsgd_set_models(wpsgd_ctx* ctx, const float* v);
+
+/* Eq. 6 / Eq. 8 weights of the last run, to weights HOST [k] (fp64), and whether the condition of
+ * Corollary 3 / 4 (Eq. 7 / Eq. 9), 2 sum_j r^{T_j} > sqrt(k) + k, holds (cond_holds may be NULL).
+ * Host-only computation; synchronous. */
+wpsgd_status wpsgd_get_weights(wpsgd_ctx* ctx, double r, double* weights, int* cond_holds);
+
+/* The weights for given step counts without a context (HOST arrays). sum_rT (may be NULL) receives
+ * sum_j r^{T_j}, the quantity in Eq. 7 / Eq. 9 and in the validity bound of averaging every span. */
+wpsgd_status wpsgd_weights(const int64_t* n_steps, int32_t k, float eta0, wpsgd_lr sched, float lambda,
+                           double r, double* weights, int* cond_holds, double* sum_rT);
+
+/* The sample stream exactly as the chain kernels draw it: row indices (within the shard of m rows)
+ * of steps n_begin+1 .. n_begin+count of node `node`, to out DEVICE [count] uint32. */
+wpsgd_status wpsgd_sample_indices(wpsgd_ctx* ctx, uint64_t seed, int32_t node, int64_t m, int64_t n_begin,
+                                  int64_t count, uint32_t* out);
+
+/* Objective of Eq. 3-4 and 0/1 error of sign(w.x) on dense rows (the paper's evaluation measures):
+ *   objective = (lambda/2)|w|^2 + mean_i L(y_i, w.x_i);  error = share of rows with sign(w.x) != sign(y).
+ *   X DEVICE [n_rows, ld_elems], y DEVICE [n_rows], w DEVICE [d]; out DEVICE [2] fp64 = {objective, error}. */
+wpsgd_status wpsgd_objective(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                             int64_t n_rows, const float* w, float lambda, wpsgd_loss loss, double* out);
+
+/* Whole path from HOST buffers: copies X HOST [N, d] (dense, contiguous), y HOST [N] and w0 HOST [d]
+ * (or NULL) to the device, runs the chains and the combination, copies v back to v_out HOST [d], and
+ * waits for completion. Page-locked host buffers give full copy speed. Device staging buffers are
+ * owned by the context and reused across calls. r as in wpsgd_combine. */
+wpsgd_status wpsgd_solve_host(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, const float* y,
+                              const int64_t* shard_off, const int64_t* n_steps, float eta0, wpsgd_lr sched,
+                              float lambda, wpsgd_loss loss, uint64_t seed, const float* w0, double r,
+                              float* v_out);
+
+/* Wait for the stream and read the device status word. WPSGD_OK, WPSGD_ERR_TIMEOUT (a bounded wait
+ * gave up), or WPSGD_ERR_CUDA (a launch or copy failed, or a kernel's own bounds check fired). */
+wpsgd_status wpsgd_check(wpsgd_ctx* ctx);
+
+/* Device time of the most recent chain kernel launch (the per-node loops only, without the sample
+ * stream kernel and the combination), in milliseconds, from events recorded on the context's
+ * stream around it. Needs wpsgd_set_option(ctx, "timing", 1) before the run; waits for the kernel. */
+wpsgd_status wpsgd_last_chain_ms(wpsgd_ctx* ctx, float* ms);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t wpsgd_launch_count(const wpsgd_ctx* ctx);
+
+/* Text of the last error on the context (or of the last context-free call when ctx is NULL).
+ * The pointer stays valid until the next call on that context. */
+const char* wpsgd_last_error(const wpsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WPSGD_H_ */

@@ -1,0 +1,68 @@
+// Sample-index stream of the chains: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11), written
+// from the published definition, and the kernel that materialises each node's stream.
+//
+// Stands for Algorithm 1's "randomly shuffle the data on machine i; get the n-th example": the
+// n-th example (1-based) of node j is row floor(u * m_j / 2^32) of its shard, u being output word
+// (n-1)&3 of the block with counter ((n-1)>>2 low, (n-1)>>2 high, j, 0) and key (seed low, seed high).
+#pragma once
+
+#include "common.cuh"
+
+namespace wpsgd {
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// Entries of steps b+1 .. b+cnt of node j (shard of m rows) into out[0 .. cnt): one counter value q
+// (four consecutive steps) per (t0 + i * stride).
+__device__ __forceinline__ void emit_indices(uint64_t seed, uint32_t j, long long b, long long cnt, uint32_t m,
+                                             uint32_t* __restrict__ out, long long t0, long long stride) {
+  const long long q_lo = b >> 2, q_hi = (b + cnt - 1) >> 2;  // zero-based step s = n-1 lies in [b, b+cnt)
+  for (long long q = q_lo + t0; q <= q_hi; q += stride) {
+    const uint4 o = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)((unsigned long long)q >> 32), j, 0u),
+                                  (uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint32_t w[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const long long s = (q << 2) + e;
+      if (s >= b && s < b + cnt) out[s - b] = __umulhi(w[e], m);  // floor(u m / 2^32)
+    }
+  }
+}
+
+// All nodes' streams for one launch of the chains. Node = blockIdx.y (+ gridDim.y per pass).
+//   idx_off[j]   position of node j's first entry in idx (prefix sums of count)
+//   first[j]     number of steps node j has already run (its entries start at step first[j]+1)
+//   count[j]     entries to produce for node j
+//   rows[j]      shard size m_j
+//   ids[j]       node number that enters the counter (j itself unless the caller renumbers nodes)
+__global__ void index_stream_kernel(uint64_t seed, int k, const long long* __restrict__ idx_off,
+                                    const long long* __restrict__ first, const long long* __restrict__ count,
+                                    const long long* __restrict__ rows, const int* __restrict__ ids,
+                                    uint32_t* __restrict__ idx) {
+  for (int j = blockIdx.y; j < k; j += gridDim.y) {
+    const long long cnt = count[j];
+    if (cnt <= 0) continue;
+    emit_indices(seed, (uint32_t)ids[j], first[j], cnt, (uint32_t)rows[j], idx + idx_off[j],
+                 (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+  }
+}
+
+// One node's stream, for callers that want to look at it.
+__global__ void index_single_kernel(uint64_t seed, int node, long long m, long long n_begin, long long count,
+                                    uint32_t* __restrict__ out) {
+  if (count > 0)
+    emit_indices(seed, (uint32_t)node, n_begin, count, (uint32_t)m, out,
+                 (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+}
+
+}  // namespace wpsgd

@@ -1,0 +1,689 @@
+// C ABI of the WP-SGD library (see include/wpsgd.h): context, host-side planning (validation,
+// delays and Eq. 6 / Eq. 8 weights in fp64, node ordering, kernel selection) and kernel launches.
+#include "../../include/wpsgd.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <numeric>
+#include <string>
+#include <vector>
+
+#include "chain_csr.cuh"
+#include "chain_dense.cuh"
+#include "combine.cuh"
+#include "philox.cuh"
+
+using namespace wpsgd;
+
+struct wpsgd_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int k = 0;
+  long long d = 0;
+  // models
+  float* W = nullptr;       // [k, d]
+  double* scale = nullptr;  // [k] (sparse path: w_j = scale_j * W[j])
+  bool scaled = false;
+  // per-launch tables on the device
+  long long* t_shard_off = nullptr;  // [k+1]
+  long long* t_steps = nullptr;      // [k]
+  long long* t_first = nullptr;      // [k]
+  long long* t_idx_off = nullptr;    // [k+1]
+  long long* t_rows = nullptr;       // [k]
+  int* t_order = nullptr;            // [k]
+  int* t_ids = nullptr;              // [k] node numbers entering the sample stream
+  double* t_weights = nullptr;       // [k]
+  uint32_t* idx = nullptr;
+  size_t idx_cap = 0;  // entries
+  DevStatus* status = nullptr;
+  double* part = nullptr;  // objective partial sums
+  size_t part_cap = 0;     // doubles
+  // staging of the host-buffer entry point
+  void* st_X = nullptr;
+  size_t st_X_cap = 0;
+  float* st_y = nullptr;
+  size_t st_y_cap = 0;
+  float* st_v = nullptr;   // [d]
+  float* st_w0 = nullptr;  // [d]
+  // state of the chains
+  bool have_run = false;
+  std::vector<long long> steps_done;
+  std::vector<int> node_ids;
+  float eta0 = 0.f, lambda = 0.f;
+  int sched = 0, loss = 0;
+  uint64_t seed = 0;
+  // options
+  int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_block_rows = 0, opt_cluster = 0, opt_sparse_threads = 32;
+  long long opt_spin_limit = 1ll << 22;
+  int opt_timing = 0;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  bool ev_valid = false;
+  long long launches = 0;
+  std::string err;
+};
+
+namespace {
+
+std::string g_err;  // last error of context-free calls
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    if (prev != dev) cudaSetDevice(dev);
+    else prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+wpsgd_status fail(wpsgd_ctx* c, wpsgd_status s, const std::string& msg) {
+  if (c) c->err = msg;
+  else g_err = msg;
+  return s;
+}
+
+#define CU_TRY(ctx, expr)                                                                          \
+  do {                                                                                             \
+    cudaError_t e_ = (expr);                                                                       \
+    if (e_ != cudaSuccess) {                                                                       \
+      const bool oom_ = (e_ == cudaErrorMemoryAllocation);                                         \
+      return fail(ctx, oom_ ? WPSGD_ERR_ALLOC : WPSGD_ERR_CUDA,                                    \
+                  std::string(#expr) + ": " + cudaGetErrorString(e_));                             \
+    }                                                                                              \
+  } while (0)
+
+template <typename T>
+wpsgd_status grow(wpsgd_ctx* c, T** p, size_t* cap, size_t need) {
+  if (need <= *cap) return WPSGD_OK;
+  if (*p) {
+    CU_TRY(c, cudaStreamSynchronize(c->stream));
+    CU_TRY(c, cudaFree(*p));
+    *p = nullptr;
+    *cap = 0;
+  }
+  const size_t want = need + need / 8;
+  void* q = nullptr;
+  CU_TRY(c, cudaMalloc(&q, want * sizeof(T)));
+  *p = (T*)q;
+  *cap = want;
+  return WPSGD_OK;
+}
+
+// ---- Eq. 6 / Eq. 8 in fp64 -------------------------------------------------------------------------
+// log of r^{T_j} (or of the product of skipped per-step factors for the decaying schedule)
+wpsgd_status log_rates(const long long* n, int k, double eta0, int sched, double lambda, double r,
+                       std::vector<double>* lg, std::string* why) {
+  long long t = 0;
+  for (int j = 0; j < k; ++j) {
+    if (n[j] < 0) {
+      *why = "negative step count";
+      return WPSGD_ERR_INVALID_ARG;
+    }
+    t = std::max(t, n[j]);
+  }
+  lg->assign(k, 0.0);
+  const bool given = r > 0.0;  // false for NaN
+  if (given) {
+    const double lr = std::log(r);
+    for (int j = 0; j < k; ++j) (*lg)[j] = (double)(t - n[j]) * lr;
+  } else if (sched == WPSGD_LR_CONST) {
+    const double lr = std::log1p(-eta0 * lambda);
+    for (int j = 0; j < k; ++j) (*lg)[j] = (double)(t - n[j]) * lr;
+  } else {
+    // sum_{s = n_j + 1}^{t} log(1 - eta_s lambda): suffix sums from the smallest n_j upward
+    long long lo = t;
+    for (int j = 0; j < k; ++j) lo = std::min(lo, n[j]);
+    std::vector<double> suf((size_t)(t - lo) + 1, 0.0);  // suf[i] = sum over s in (lo + i, t]
+    for (long long s = t; s > lo; --s)
+      suf[(size_t)(s - 1 - lo)] = suf[(size_t)(s - lo)] + std::log1p(-eta0 / std::sqrt((double)s) * lambda);
+    for (int j = 0; j < k; ++j) (*lg)[j] = suf[(size_t)(n[j] - lo)];
+  }
+  return WPSGD_OK;
+}
+
+wpsgd_status weights_host(const long long* n, int k, float eta0, int sched, float lambda, double r, double* w,
+                          int* cond, double* sum_rT, std::string* why) {
+  if (!n || !w || k < 1) {
+    *why = "weights: null argument or k < 1";
+    return WPSGD_ERR_INVALID_ARG;
+  }
+  if (sched != WPSGD_LR_CONST && sched != WPSGD_LR_INV_SQRT) {
+    *why = "weights: unknown schedule";
+    return WPSGD_ERR_INVALID_ARG;
+  }
+  std::vector<double> lg;
+  wpsgd_status s = log_rates(n, k, (double)eta0, sched, (double)lambda, r, &lg, why);
+  if (s != WPSGD_OK) return s;
+  const double mx = *std::max_element(lg.begin(), lg.end());
+  double tot = 0.0, tot_raw = 0.0;
+  for (int j = 0; j < k; ++j) {
+    tot += std::exp(lg[j] - mx);
+    tot_raw += std::exp(lg[j]);
+  }
+  for (int j = 0; j < k; ++j) w[j] = std::exp(lg[j] - mx) / tot;
+  if (sum_rT) *sum_rT = tot_raw;
+  if (cond) *cond = (2.0 * tot_raw > std::sqrt((double)k) + (double)k) ? 1 : 0;
+  return WPSGD_OK;
+}
+
+int grid_for(long long work_items, int block, int cap = 148 * 16) {
+  long long g = (work_items + block - 1) / block;
+  return (int)std::max(1ll, std::min<long long>(g, cap));
+}
+
+// ---- common part of run / continue: tables, sample stream ---------------------------------------------
+struct Plan {
+  std::vector<long long> off, steps, first, idx_off, rows;
+  std::vector<int> order;
+  long long total = 0;
+};
+
+wpsgd_status make_plan(wpsgd_ctx* c, const long long* shard_off, const long long* n_steps,
+                       const std::vector<long long>& first, Plan* pl) {
+  const int k = c->k;
+  if (!shard_off || !n_steps) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off / n_steps is NULL");
+  if (shard_off[0] < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off[0] < 0");
+  pl->off.assign(shard_off, shard_off + k + 1);
+  pl->steps.assign(n_steps, n_steps + k);
+  pl->first = first;
+  pl->idx_off.assign(k + 1, 0);
+  pl->rows.assign(k, 0);
+  for (int j = 0; j < k; ++j) {
+    const long long m = shard_off[j + 1] - shard_off[j];
+    if (m < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off is not non-decreasing");
+    if (n_steps[j] < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "negative step count");
+    if (n_steps[j] > 0 && m < 1) return fail(c, WPSGD_ERR_INVALID_ARG, "a node with steps has an empty shard");
+    if (m > 0xFFFFFFFFll) return fail(c, WPSGD_ERR_INVALID_ARG, "a shard has 2^32 rows or more");
+    pl->rows[j] = m;
+    pl->idx_off[j + 1] = pl->idx_off[j] + n_steps[j];
+  }
+  pl->total = pl->idx_off[k];
+  pl->order.resize(k);
+  std::iota(pl->order.begin(), pl->order.end(), 0);
+  std::stable_sort(pl->order.begin(), pl->order.end(), [&](int a, int b) { return n_steps[a] > n_steps[b]; });
+  return WPSGD_OK;
+}
+
+wpsgd_status upload_plan_and_stream(wpsgd_ctx* c, const Plan& pl) {
+  const int k = c->k;
+  wpsgd_status s = grow(c, &c->idx, &c->idx_cap, (size_t)std::max(1ll, pl.total));
+  if (s != WPSGD_OK) return s;
+  // pageable sources: the copy has left the host buffer when cudaMemcpyAsync returns
+  CU_TRY(c, cudaMemcpyAsync(c->t_shard_off, pl.off.data(), (k + 1) * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_steps, pl.steps.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_first, pl.first.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_idx_off, pl.idx_off.data(), (k + 1) * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_rows, pl.rows.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_order, pl.order.data(), k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_ids, c->node_ids.data(), k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  if (pl.total > 0) {
+    const long long longest = *std::max_element(pl.steps.begin(), pl.steps.end());
+    dim3 grid((unsigned)grid_for((longest + 3) / 4 + 1, 256, 1024), (unsigned)std::min(k, 65535));
+    index_stream_kernel<<<grid, 256, 0, c->stream>>>(c->seed, k, c->t_idx_off, c->t_first, c->t_steps, c->t_rows, c->t_ids, c->idx);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+  }
+  return WPSGD_OK;
+}
+
+wpsgd_status check_hyper(wpsgd_ctx* c, float eta0, int sched, float lambda, int loss) {
+  if (!(eta0 >= 0.0f) || !std::isfinite(eta0)) return fail(c, WPSGD_ERR_INVALID_ARG, "eta0 must be finite and >= 0");
+  if (!(lambda >= 0.0f) || !std::isfinite(lambda)) return fail(c, WPSGD_ERR_INVALID_ARG, "lambda must be finite and >= 0");
+  if (!((double)eta0 * (double)lambda < 1.0)) return fail(c, WPSGD_ERR_INVALID_ARG, "eta * lambda must be < 1");
+  if (sched != WPSGD_LR_CONST && sched != WPSGD_LR_INV_SQRT) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown schedule");
+  if (loss < 0 || loss > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown loss");
+  return WPSGD_OK;
+}
+
+wpsgd_status timing_begin(wpsgd_ctx* c) {
+  c->ev_valid = false;
+  if (!c->opt_timing) return WPSGD_OK;
+  if (!c->ev0) {
+    CU_TRY(c, cudaEventCreate(&c->ev0));
+    CU_TRY(c, cudaEventCreate(&c->ev1));
+  }
+  CU_TRY(c, cudaEventRecord(c->ev0, c->stream));
+  return WPSGD_OK;
+}
+
+wpsgd_status timing_end(wpsgd_ctx* c) {
+  if (!c->opt_timing) return WPSGD_OK;
+  CU_TRY(c, cudaEventRecord(c->ev1, c->stream));
+  c->ev_valid = true;
+  return WPSGD_OK;
+}
+
+// ---- dense chain launch ---------------------------------------------------------------------------------
+template <typename XT, int R, int PF>
+wpsgd_status launch_reg(wpsgd_ctx* c, const ChainParams& p, bool block_per_node, int threads) {
+  if (block_per_node) {
+    chain_reg_kernel<XT, R, PF, true><<<c->k, threads, 0, c->stream>>>(p);
+  } else {
+    const int nodes_per_cta = 4;
+    chain_reg_kernel<XT, R, PF, false><<<(c->k + nodes_per_cta - 1) / nodes_per_cta, 32 * nodes_per_cta, 0, c->stream>>>(p);
+  }
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+template <typename XT, int R>
+wpsgd_status launch_reg_pf(wpsgd_ctx* c, const ChainParams& p, bool bpn, int threads, int pf) {
+  switch (pf) {
+    case 2: return launch_reg<XT, R, 2>(c, p, bpn, threads);
+    case 4: return launch_reg<XT, R, 4>(c, p, bpn, threads);
+    default: return launch_reg<XT, R, 8>(c, p, bpn, threads);
+  }
+}
+
+template <typename XT>
+wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
+  constexpr int V = XVec<XT>::V;
+  const long long d = c->d;
+  const bool aligned = ((uintptr_t)p.X % 16 == 0) && ((p.ld * (long long)sizeof(XT)) % 16 == 0) && (d % V == 0) &&
+                       ((uintptr_t)c->W % 16 == 0);
+  const long long chunks = d / V;
+  int variant = c->opt_variant;
+  if (variant == 0) {
+    if (!aligned || chunks > 512 * 4) variant = 1;
+    else variant = (chunks <= 64) ? 3 : 2;
+  }
+  if ((variant == 2 || variant == 3) && !aligned)
+    return fail(c, WPSGD_ERR_UNSUPPORTED, "register kernels need 16-byte aligned rows and d a multiple of 16 bytes");
+  if (variant == 3 && chunks > 32 * 4) return fail(c, WPSGD_ERR_UNSUPPORTED, "warp-per-node kernel: d too large");
+  if (variant == 2 && chunks > 512 * 4) return fail(c, WPSGD_ERR_UNSUPPORTED, "CTA-per-node kernel: d too large");
+  if (variant == 1) {
+    chain_generic_kernel<XT><<<c->k, 256, 0, c->stream>>>(p);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+    return WPSGD_OK;
+  }
+  if (variant != 2 && variant != 3) return fail(c, WPSGD_ERR_UNSUPPORTED, "dense_variant not available");
+  int threads = 32, R = 1;
+  if (variant == 3) {
+    R = (int)((chunks + 31) / 32);
+  } else {
+    threads = c->opt_threads > 0 ? c->opt_threads : (int)std::min<long long>(512, ((chunks + 31) / 32) * 32);
+    R = (int)((chunks + threads - 1) / threads);
+  }
+  if (R > 2) R = 4;  // instantiated: 1, 2, 4
+  if ((long long)R * threads < chunks) return fail(c, WPSGD_ERR_UNSUPPORTED, "threads too few for d");
+  int pf = c->opt_prefetch > 0 ? c->opt_prefetch : std::max(2, 8 / R);
+  pf = pf >= 8 ? 8 : (pf >= 4 ? 4 : 2);
+  const bool bpn = variant == 2;
+  switch (R) {
+    case 1: return launch_reg_pf<XT, 1>(c, p, bpn, threads, pf);
+    case 2: return launch_reg_pf<XT, 2>(c, p, bpn, threads, pf);
+    default: return launch_reg_pf<XT, 4>(c, p, bpn, threads, pf);
+  }
+}
+
+wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long long ld, const float* y,
+                              const long long* shard_off, const long long* n_steps, const float* w0, bool resume) {
+  if (xt != WPSGD_X_F32 && xt != WPSGD_X_BF16) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown feature type");
+  if (ld < c->d) return fail(c, WPSGD_ERR_INVALID_ARG, "ld_elems < d");
+  Plan pl;
+  std::vector<long long> first = resume ? c->steps_done : std::vector<long long>(c->k, 0);
+  wpsgd_status s = make_plan(c, (const long long*)shard_off, (const long long*)n_steps, first, &pl);
+  if (s != WPSGD_OK) return s;
+  if (pl.total > 0 && (!X || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "X or y is NULL");
+  s = upload_plan_and_stream(c, pl);
+  if (s != WPSGD_OK) return s;
+  ChainParams p;
+  p.X = X; p.ld = ld; p.y = y;
+  p.shard_off = c->t_shard_off; p.n_steps = c->t_steps; p.first = c->t_first; p.idx_off = c->t_idx_off;
+  p.idx = c->idx; p.order = c->t_order; p.W = c->W; p.w0 = w0; p.resume = resume ? 1 : 0;
+  p.k = c->k; p.d = c->d; p.eta0 = c->eta0; p.sched = c->sched; p.lambda = c->lambda; p.loss = c->loss;
+  p.status = c->status;
+  s = timing_begin(c);
+  if (s != WPSGD_OK) return s;
+  s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, p) : launch_dense<__nv_bfloat16>(c, p);
+  if (s != WPSGD_OK) return s;
+  s = timing_end(c);
+  if (s != WPSGD_OK) return s;
+  for (int j = 0; j < c->k; ++j) c->steps_done[j] = first[j] + n_steps[j];
+  c->have_run = true;
+  c->scaled = false;
+  return WPSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, wpsgd_ctx** out) {
+  if (!out) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (k < 1 || d < 1) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "k and d must be >= 1");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    return fail(nullptr, WPSGD_ERR_CUDA, "no CUDA device available");
+  }
+  if (device < 0 || device >= ndev) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "device index out of range");
+  DeviceGuard guard(device);
+  wpsgd_ctx* c = new wpsgd_ctx();
+  c->device = device;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->k = k;
+  c->d = d;
+  c->steps_done.assign(k, 0);
+  c->node_ids.resize(k);
+  std::iota(c->node_ids.begin(), c->node_ids.end(), 0);
+  auto bail = [&](cudaError_t e, const char* what) {
+    g_err = std::string(what) + ": " + cudaGetErrorString(e);
+    const wpsgd_status s = (e == cudaErrorMemoryAllocation) ? WPSGD_ERR_ALLOC : WPSGD_ERR_CUDA;
+    cudaGetLastError();
+    wpsgd_destroy(c);
+    return s;
+  };
+  cudaError_t e;
+#define ALLOC(ptr, bytes)                                         \
+  if ((e = cudaMalloc((void**)&(ptr), (bytes))) != cudaSuccess) return bail(e, "cudaMalloc(" #ptr ")");
+  ALLOC(c->W, (size_t)k * (size_t)d * sizeof(float));
+  ALLOC(c->scale, (size_t)k * sizeof(double));
+  ALLOC(c->t_shard_off, (size_t)(k + 1) * sizeof(long long));
+  ALLOC(c->t_steps, (size_t)k * sizeof(long long));
+  ALLOC(c->t_first, (size_t)k * sizeof(long long));
+  ALLOC(c->t_idx_off, (size_t)(k + 1) * sizeof(long long));
+  ALLOC(c->t_rows, (size_t)k * sizeof(long long));
+  ALLOC(c->t_order, (size_t)k * sizeof(int));
+  ALLOC(c->t_ids, (size_t)k * sizeof(int));
+  ALLOC(c->t_weights, (size_t)k * sizeof(double));
+  ALLOC(c->status, sizeof(DevStatus));
+#undef ALLOC
+  if ((e = cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
+  *out = c;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_destroy(wpsgd_ctx* c) {
+  if (!c) return WPSGD_OK;
+  DeviceGuard guard(c->device);
+  cudaStreamSynchronize(c->stream);
+  void* ptrs[] = {c->W, c->scale, c->t_shard_off, c->t_steps, c->t_first, c->t_idx_off, c->t_rows, c->t_order,
+                  c->t_ids, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+  cudaGetLastError();
+  delete c;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
+  if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
+  const std::string n(name);
+  if (n == "dense_variant") {
+    if (value < 0 || value > 4) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..4");
+    c->opt_variant = (int)value;
+  } else if (n == "prefetch") {
+    if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");
+    c->opt_prefetch = (int)value;
+  } else if (n == "threads") {
+    if (value != 0 && (value < 32 || value > 512 || value % 32)) return fail(c, WPSGD_ERR_INVALID_ARG, "threads must be 0 or a multiple of 32 in 32..512");
+    c->opt_threads = (int)value;
+  } else if (n == "block_rows") {
+    if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "block_rows must be 0..64");
+    c->opt_block_rows = (int)value;
+  } else if (n == "cluster") {
+    if (value < 0 || value > 16) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0..16");
+    c->opt_cluster = (int)value;
+  } else if (n == "sparse_threads") {
+    if (value != 32) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_threads must be 32");
+    c->opt_sparse_threads = (int)value;
+  } else if (n == "timing") {
+    if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "timing must be 0 or 1");
+    c->opt_timing = (int)value;
+  } else if (n == "spin_limit") {
+    if (value < 1) return fail(c, WPSGD_ERR_INVALID_ARG, "spin_limit must be >= 1");
+    c->opt_spin_limit = value;
+  } else {
+    return fail(c, WPSGD_ERR_INVALID_ARG, "unknown option: " + n);
+  }
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_set_node_ids(wpsgd_ctx* c, const int32_t* ids) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!ids) {
+    std::iota(c->node_ids.begin(), c->node_ids.end(), 0);
+    return WPSGD_OK;
+  }
+  for (int j = 0; j < c->k; ++j)
+    if (ids[j] < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "node ids must be >= 0");
+  c->node_ids.assign(ids, ids + c->k);
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_run(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                       const int64_t* shard_off, const int64_t* n_steps, float eta0, wpsgd_lr sched, float lambda,
+                       wpsgd_loss loss, uint64_t seed, const float* w0) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  wpsgd_status s = check_hyper(c, eta0, (int)sched, lambda, (int)loss);
+  if (s != WPSGD_OK) return s;
+  c->eta0 = eta0; c->sched = (int)sched; c->lambda = lambda; c->loss = (int)loss; c->seed = seed;
+  c->have_run = false;
+  return run_dense_common(c, X, xt, ld_elems, y, (const long long*)shard_off, (const long long*)n_steps, w0, false);
+}
+
+wpsgd_status wpsgd_continue(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                            const int64_t* shard_off, const int64_t* n_more) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "continue before run");
+  if (c->scaled) return fail(c, WPSGD_ERR_UNSUPPORTED, "continue is available for dense data only");
+  DeviceGuard guard(c->device);
+  return run_dense_common(c, X, xt, ld_elems, y, (const long long*)shard_off, (const long long*)n_more, nullptr, true);
+}
+
+wpsgd_status wpsgd_run_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                           const float* y, const int64_t* shard_off, const int64_t* n_steps, float eta0,
+                           wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed, const float* w0) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  wpsgd_status s = check_hyper(c, eta0, (int)sched, lambda, (int)loss);
+  if (s != WPSGD_OK) return s;
+  c->eta0 = eta0; c->sched = (int)sched; c->lambda = lambda; c->loss = (int)loss; c->seed = seed;
+  c->have_run = false;
+  Plan pl;
+  s = make_plan(c, (const long long*)shard_off, (const long long*)n_steps, std::vector<long long>(c->k, 0), &pl);
+  if (s != WPSGD_OK) return s;
+  if (pl.total > 0 && (!row_ptr || !col_idx || !val || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "a CSR array or y is NULL");
+  s = upload_plan_and_stream(c, pl);
+  if (s != WPSGD_OK) return s;
+  csr_init_kernel<<<grid_for((long long)c->k * c->d, 256), 256, 0, c->stream>>>(c->W, c->scale, w0, c->k, c->d);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  CsrParams p;
+  p.row_ptr = (const long long*)row_ptr; p.col_idx = col_idx; p.val = val; p.y = y;
+  p.shard_off = c->t_shard_off; p.n_steps = c->t_steps; p.idx_off = c->t_idx_off; p.idx = c->idx;
+  p.order = c->t_order; p.U = c->W; p.scale = c->scale; p.k = c->k; p.d = c->d;
+  p.eta0 = eta0; p.sched = (int)sched; p.lambda = lambda; p.loss = (int)loss; p.status = c->status;
+  s = timing_begin(c);
+  if (s != WPSGD_OK) return s;
+  const int pf = c->opt_prefetch > 0 ? c->opt_prefetch : 4;
+  if (pf >= 8) chain_csr_kernel<8><<<c->k, 32, 0, c->stream>>>(p);
+  else if (pf >= 4) chain_csr_kernel<4><<<c->k, 32, 0, c->stream>>>(p);
+  else chain_csr_kernel<2><<<c->k, 32, 0, c->stream>>>(p);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  s = timing_end(c);
+  if (s != WPSGD_OK) return s;
+  for (int j = 0; j < c->k; ++j) c->steps_done[j] = n_steps[j];
+  c->have_run = true;
+  c->scaled = true;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_get_weights(wpsgd_ctx* c, double r, double* weights, int* cond_holds) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "weights before run");
+  std::string why;
+  wpsgd_status s = weights_host(c->steps_done.data(), c->k, c->eta0, c->sched, c->lambda, r, weights, cond_holds, nullptr, &why);
+  return s == WPSGD_OK ? s : fail(c, s, why);
+}
+
+wpsgd_status wpsgd_weights(const int64_t* n_steps, int32_t k, float eta0, wpsgd_lr sched, float lambda, double r,
+                           double* weights, int* cond_holds, double* sum_rT) {
+  std::string why;
+  wpsgd_status s = weights_host((const long long*)n_steps, k, eta0, (int)sched, lambda, r, weights, cond_holds, sum_rT, &why);
+  return s == WPSGD_OK ? s : fail(nullptr, s, why);
+}
+
+wpsgd_status wpsgd_combine(wpsgd_ctx* c, double r, float* v_out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "combine before run");
+  if (!v_out) return fail(c, WPSGD_ERR_INVALID_ARG, "v_out is NULL");
+  DeviceGuard guard(c->device);
+  std::vector<double> w(c->k);
+  std::string why;
+  wpsgd_status s = weights_host(c->steps_done.data(), c->k, c->eta0, c->sched, c->lambda, r, w.data(), nullptr, nullptr, &why);
+  if (s != WPSGD_OK) return fail(c, s, why);
+  CU_TRY(c, cudaMemcpyAsync(c->t_weights, w.data(), c->k * sizeof(double), cudaMemcpyHostToDevice, c->stream));
+  combine_kernel<<<grid_for(c->d, 256), 256, 0, c->stream>>>(c->W, c->t_weights, c->scaled ? c->scale : nullptr, c->k,
+                                                            c->d, v_out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_combine_weighted(wpsgd_ctx* c, const double* weights, float* v_out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "combine before run");
+  if (!v_out || !weights) return fail(c, WPSGD_ERR_INVALID_ARG, "weights or v_out is NULL");
+  for (int j = 0; j < c->k; ++j)
+    if (!std::isfinite(weights[j])) return fail(c, WPSGD_ERR_INVALID_ARG, "a weight is not finite");
+  DeviceGuard guard(c->device);
+  CU_TRY(c, cudaMemcpyAsync(c->t_weights, weights, c->k * sizeof(double), cudaMemcpyHostToDevice, c->stream));
+  combine_kernel<<<grid_for(c->d, 256), 256, 0, c->stream>>>(c->W, c->t_weights, c->scaled ? c->scale : nullptr, c->k,
+                                                            c->d, v_out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_last_chain_ms(wpsgd_ctx* c, float* ms) {
+  if (!c || !ms) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or ms is NULL");
+  if (!c->ev_valid) return fail(c, WPSGD_ERR_STATE, "no timed chain launch (set option \"timing\" to 1 before the run)");
+  DeviceGuard guard(c->device);
+  CU_TRY(c, cudaEventSynchronize(c->ev1));
+  CU_TRY(c, cudaEventElapsedTime(ms, c->ev0, c->ev1));
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_get_models(wpsgd_ctx* c, float* W_out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "get_models before run");
+  if (!W_out) return fail(c, WPSGD_ERR_INVALID_ARG, "W_out is NULL");
+  DeviceGuard guard(c->device);
+  export_models_kernel<<<grid_for((long long)c->k * c->d, 256), 256, 0, c->stream>>>(
+      c->W, c->scaled ? c->scale : nullptr, c->k, c->d, W_out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_set_models(wpsgd_ctx* c, const float* v) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "set_models before run");
+  if (!v) return fail(c, WPSGD_ERR_INVALID_ARG, "v is NULL");
+  DeviceGuard guard(c->device);
+  broadcast_model_kernel<<<grid_for((long long)c->k * c->d, 256), 256, 0, c->stream>>>(c->W, c->scale, v, c->k, c->d);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_sample_indices(wpsgd_ctx* c, uint64_t seed, int32_t node, int64_t m, int64_t n_begin, int64_t count,
+                                  uint32_t* out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (node < 0 || m < 1 || m > 0xFFFFFFFFll || n_begin < 0 || count < 0)
+    return fail(c, WPSGD_ERR_INVALID_ARG, "sample_indices: need node >= 0, 1 <= m < 2^32, n_begin >= 0, count >= 0");
+  if (count == 0) return WPSGD_OK;
+  if (!out) return fail(c, WPSGD_ERR_INVALID_ARG, "out is NULL");
+  DeviceGuard guard(c->device);
+  index_single_kernel<<<grid_for((count + 3) / 4 + 1, 256), 256, 0, c->stream>>>(seed, node, m, n_begin, count, out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_objective(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
+                             int64_t n_rows, const float* w, float lambda, wpsgd_loss loss, double* out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!w || !out || n_rows < 0 || ld_elems < c->d || (int)loss < 0 || (int)loss > 2 || (n_rows > 0 && (!X || !y)))
+    return fail(c, WPSGD_ERR_INVALID_ARG, "objective: bad argument");
+  if (xt != WPSGD_X_F32 && xt != WPSGD_X_BF16) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown feature type");
+  DeviceGuard guard(c->device);
+  const int nblk = grid_for((n_rows + 7) / 8, 1, 148 * 8);
+  wpsgd_status s = grow(c, &c->part, &c->part_cap, (size_t)nblk * 2);
+  if (s != WPSGD_OK) return s;
+  if (xt == WPSGD_X_F32)
+    objective_rows_kernel<float><<<nblk, 256, 0, c->stream>>>((const float*)X, ld_elems, y, n_rows, w, c->d, (int)loss, c->part);
+  else
+    objective_rows_kernel<__nv_bfloat16><<<nblk, 256, 0, c->stream>>>((const __nv_bfloat16*)X, ld_elems, y, n_rows, w, c->d, (int)loss, c->part);
+  CU_TRY(c, cudaGetLastError());
+  objective_finish_kernel<<<1, 256, 0, c->stream>>>(c->part, nblk, w, c->d, lambda, n_rows, out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches += 2;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_solve_host(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, const float* y, const int64_t* shard_off,
+                              const int64_t* n_steps, float eta0, wpsgd_lr sched, float lambda, wpsgd_loss loss,
+                              uint64_t seed, const float* w0, double r, float* v_out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!shard_off || !v_out) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off or v_out is NULL");
+  if (xt != WPSGD_X_F32 && xt != WPSGD_X_BF16) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown feature type");
+  DeviceGuard guard(c->device);
+  const long long N = shard_off[c->k];
+  if (N < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off[k] < 0");
+  if (N > 0 && (!X || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "X or y is NULL");
+  const size_t es = xt == WPSGD_X_F32 ? 4 : 2;
+  const size_t xbytes = (size_t)N * (size_t)c->d * es;
+  char* sx = (char*)c->st_X;
+  wpsgd_status s = grow(c, &sx, &c->st_X_cap, std::max<size_t>(xbytes, 16));
+  c->st_X = sx;
+  if (s != WPSGD_OK) return s;
+  s = grow(c, &c->st_y, &c->st_y_cap, (size_t)std::max(1ll, N));
+  if (s != WPSGD_OK) return s;
+  if (!c->st_v) CU_TRY(c, cudaMalloc((void**)&c->st_v, (size_t)c->d * sizeof(float)));
+  if (w0 && !c->st_w0) CU_TRY(c, cudaMalloc((void**)&c->st_w0, (size_t)c->d * sizeof(float)));
+  if (N > 0) {
+    CU_TRY(c, cudaMemcpyAsync(c->st_X, X, xbytes, cudaMemcpyHostToDevice, c->stream));
+    CU_TRY(c, cudaMemcpyAsync(c->st_y, y, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  }
+  if (w0) CU_TRY(c, cudaMemcpyAsync(c->st_w0, w0, (size_t)c->d * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  s = wpsgd_run(c, c->st_X, xt, c->d, c->st_y, shard_off, n_steps, eta0, sched, lambda, loss, seed, w0 ? c->st_w0 : nullptr);
+  if (s != WPSGD_OK) return s;
+  s = wpsgd_combine(c, r, c->st_v);
+  if (s != WPSGD_OK) return s;
+  CU_TRY(c, cudaMemcpyAsync(v_out, c->st_v, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(c, cudaStreamSynchronize(c->stream));
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_check(wpsgd_ctx* c) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  DevStatus h;
+  CU_TRY(c, cudaMemcpyAsync(&h, c->status, sizeof(h), cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(c, cudaStreamSynchronize(c->stream));
+  if (h.code == DEV_OK) return WPSGD_OK;
+  char buf[160];
+  snprintf(buf, sizeof(buf), "device status %d at %d (detail %lld)", h.code, h.where, h.detail);
+  cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream);
+  return fail(c, h.code == DEV_TIMEOUT ? WPSGD_ERR_TIMEOUT : WPSGD_ERR_CUDA, buf);
+}
+
+int64_t wpsgd_launch_count(const wpsgd_ctx* c) { return c ? c->launches : 0; }
+
+const char* wpsgd_last_error(const wpsgd_ctx* c) { return c ? c->err.c_str() : g_err.c_str(); }
+
+}  // extern "C"

@@ -25,3 +25,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session")
+def wpsgd_lib():
+    """The built C-ABI library (compiled on demand with nvcc; no GPU needed to build)."""
+    from paper_1708_04801_b200 import build as _b
+
+    _b.build()
+    import paper_1708_04801_b200 as P
+
+    return P.load_library()

@@ -1,0 +1,347 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs. Sample streams bit-exact; models within relative L2 error 1e-4 (logistic, squared)
+or 1e-3 (hinge: a margin within rounding of 1 may flip one subgradient)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import wpsgd_inputs as wi
+
+pytestmark = pytest.mark.gpu
+
+HINGE, LOGISTIC, SQUARED = 0, 1, 2
+TOL = {HINGE: 1e-3, LOGISTIC: 1e-4, SQUARED: 1e-4}
+
+
+@pytest.fixture(scope="module")
+def P(wpsgd_lib):
+    import paper_1708_04801_b200 as pkg
+
+    return pkg
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    den = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a))
+
+
+def gpu_solve(P, wl_cpu, options=None, r=0.0):
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        for k_, v_ in (options or {}).items():
+            ctx.set_option(k_, v_)
+        ctx.run_workload(wl)
+        v = ctx.combine(r)
+        W = ctx.get_models()
+        wts, flag = ctx.get_weights(r)
+        ctx.check()
+        return v.cpu().numpy(), W.cpu().numpy(), wts, flag
+
+
+def assert_parity(P, wl, options=None, r=0.0, tol=None):
+    v, W, wts, flag = gpu_solve(P, wl, options, r)
+    ov, oW, owts = oracle.solve(wl, r)
+    tol = tol or TOL[wl.loss]
+    np.testing.assert_allclose(wts, owts, rtol=1e-12)
+    worst = max(rel_l2(W[j], oW[j]) for j in range(wl.k) if np.linalg.norm(oW[j]) > 0)
+    assert worst <= tol, f"per-node model error {worst:.3e} > {tol}"
+    err = rel_l2(v, ov)
+    assert err <= tol, f"combined model error {err:.3e} > {tol}"
+    return err
+
+
+# ---- sample stream ------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,node,m,n_begin,count", [
+    (0, 0, 4096, 0, 1000), (0, 3, 4096, 0, 250), (1, 15, 8192, 0, 20001), (7, 2, 1, 0, 17),
+    (0xFFFFFFFFFFFFFFFF, 1023, (1 << 32) - 1, 0, 4099), (5, 9, 65536, 1, 1), (5, 9, 65536, 2, 3), (5, 9, 65536, 3, 6),
+    (5, 9, 65536, 1237, 3763), (0x123456789ABCDEF1, 77, 2047, 999999999, 1025), (3, 1, 10, 0, 0),
+    (2, 4, 3, (1 << 34) + 1, 13),
+])
+def test_sample_stream_bit_exact(P, seed, node, m, n_begin, count):
+    with P.Context(2, 8) as ctx:
+        got = ctx.sample_indices(seed, node, m, n_begin, count).cpu().numpy().view(np.uint32)
+        ctx.check()
+    want = oracle.sample_indices(seed, node, m, n_begin, count)
+    assert np.array_equal(got, want)
+
+
+# ---- the five workloads, scaled down, default kernel choice ---------------------------------------------
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_small_workloads_default_kernels(P, cfg):
+    assert_parity(P, wi.small(cfg))
+
+
+# ---- every dense kernel variant ----------------------------------------------------------------------
+@pytest.mark.parametrize("variant,threads,prefetch", [(1, 0, 0), (2, 0, 2), (2, 0, 4), (2, 0, 8), (2, 128, 4), (2, 64, 8),
+                                                      (2, 32, 2), (3, 0, 2), (3, 0, 4), (3, 0, 8)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_dense_variants(P, variant, threads, prefetch, bf16):
+    # d = 480: 120 fp32 / 60 bf16 16-byte chunks: ragged against 32-lane and 128-thread tiles
+    wl = wi.config2(k=5, d=480, m=96, base_steps=333)
+    if bf16:
+        wl.X = wl.X.to(torch.bfloat16)
+    assert_parity(P, wl, {"dense_variant": variant, "threads": threads, "prefetch": prefetch})
+
+
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("sched", [0, 1])
+@pytest.mark.parametrize("variant", [1, 2, 3])
+def test_losses_and_schedules(P, loss, sched, variant):
+    wl = wi.config1(k=3, d=64, m=128, n_steps=(300, 150, 40))
+    wl.loss, wl.sched = loss, sched
+    wl.eta0 = 0.05 if sched else 0.01
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.5 + 0.1).contiguous()
+    assert_parity(P, wl, {"dense_variant": variant})
+
+
+def test_generic_kernel_handles_unaligned_shapes(P):
+    # d = 67 (not a multiple of 4), row stride 71: only the generic kernel applies, and auto must pick it
+    g = torch.Generator().manual_seed(3)
+    k, d, ld, m = 3, 67, 71, 50
+    Xp = torch.randn(k * m, ld, generator=g) / 8
+    y = torch.sign(torch.randn(k * m, generator=g))
+    off = np.arange(k + 1, dtype=np.int64) * m
+    n = np.array([200, 77, 0], dtype=np.int64)
+    oW = oracle.run_dense(Xp, y, off, n, d, 0.05, 0, 1e-2, LOGISTIC, 11)
+    Xd = Xp.cuda()
+    with P.Context(k, d) as ctx:
+        ctx.run(Xd[:, :d], y.cuda(), off, n, 0.05, 0, 1e-2, LOGISTIC, 11)
+        W = ctx.get_models().cpu().numpy()
+        ctx.check()
+        with pytest.raises(P.WpsgdError) as e:
+            ctx.set_option("dense_variant", 2)
+            ctx.run(Xd[:, :d], y.cuda(), off, n, 0.05, 0, 1e-2, LOGISTIC, 11)
+        assert e.value.status_name == "UNSUPPORTED"
+    for j in range(2):
+        assert rel_l2(W[j], oW[j]) <= 1e-4
+    assert np.all(W[2] == 0)
+
+
+def test_large_d_falls_back_and_matches(P):
+    wl = wi.config2(k=2, d=8200, m=16, base_steps=40)  # beyond the register kernels' reach
+    assert_parity(P, wl)
+
+
+# ---- degenerate cases -----------------------------------------------------------------------------------
+def test_nodes_without_work_keep_w0(P):
+    wl = wi.config1(k=4, d=64, m=64, n_steps=(120, 0, 30, 0))
+    wl.w0 = torch.full((64,), 4.0)  # the paper's experiments start from the constant vector 4
+    v, W, wts, _ = gpu_solve(P, wl)
+    assert np.all(W[1] == 4.0) and np.all(W[3] == 4.0)
+    assert_parity(P, wl)
+
+
+def test_no_work_at_all_returns_w0(P):
+    wl = wi.config1(k=3, d=64, m=8, n_steps=(0, 0, 0))
+    wl.w0 = torch.arange(64, dtype=torch.float32)
+    v, W, wts, _ = gpu_solve(P, wl)
+    np.testing.assert_array_equal(wts, np.full(3, 1 / 3))
+    np.testing.assert_allclose(v, np.arange(64), rtol=1e-6)
+    wl.w0 = None
+    v, W, _, _ = gpu_solve(P, wl)
+    assert np.all(v == 0) and np.all(W == 0)
+
+
+def test_single_node_is_sequential_sgd(P):
+    wl = wi.config1(k=1, d=64, m=256, n_steps=(500,))
+    v, W, wts, flag = gpu_solve(P, wl)
+    assert wts[0] == 1.0 and flag is False  # Eq. 7 with k = 1: 2 > 2 is false
+    np.testing.assert_array_equal(v, W[0])
+    assert_parity(P, wl)
+
+
+def test_single_row_shards_and_unequal_shards(P):
+    g = torch.Generator().manual_seed(5)
+    d = 32
+    off = np.array([0, 1, 4, 4, 40], dtype=np.int64)  # shard sizes 1, 3, 0, 36
+    X = torch.randn(40, d, generator=g) / 4
+    y = torch.sign(torch.randn(40, generator=g))
+    n = np.array([25, 60, 0, 100], dtype=np.int64)
+    wl = wi.Workload("ragged", 4, d, off, n, 0.05, 0, 0.01, LOGISTIC, 9, y, X=X)
+    assert_parity(P, wl)
+    for variant in (1, 2, 3):
+        assert_parity(P, wl, {"dense_variant": variant})
+
+
+def test_equal_work_reduces_to_plain_average(P):
+    wl = wi.config2(k=6, d=128, m=64, base_steps=90)
+    wl.n_steps[:] = 90
+    v, W, wts, _ = gpu_solve(P, wl)
+    np.testing.assert_array_equal(wts, np.full(6, 1 / 6))
+    np.testing.assert_allclose(v, W.astype(np.float64).mean(0), rtol=1e-6, atol=1e-9)
+
+
+def test_relabelling_a_node_changes_only_its_stream(P):
+    # the same shard at node position j must see the oracle's stream for node j
+    wl = wi.config1(k=3, d=64, m=64, n_steps=(50, 50, 50))
+    _, W, _, _ = gpu_solve(P, wl)
+    assert not np.array_equal(W[0], W[1])
+    assert_parity(P, wl)
+
+
+# ---- combination --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("r", [0.0, 1.0, 0.99999, 0.9])
+def test_combine_rates(P, r):
+    wl = wi.config1(k=4, d=64, m=64, n_steps=(400, 300, 100, 7))
+    v, W, wts, flag = gpu_solve(P, wl, r=r)
+    owts, oflag, _ = oracle.weights(wl.n_steps, wl.eta0, wl.sched, wl.lam, r)
+    np.testing.assert_allclose(wts, owts, rtol=1e-12)
+    assert flag == oflag
+    want = oracle.combine(W.astype(np.float64), owts)  # the GPU's own models, so this isolates the reduction
+    np.testing.assert_allclose(v, want, rtol=2e-7, atol=1e-12)
+
+
+def test_combine_many_nodes_ragged_d(P):
+    k, d = 37, 1001
+    g = torch.Generator().manual_seed(1)
+    X = torch.randn(k * 4, d, generator=g)
+    y = torch.sign(torch.randn(k * 4, generator=g))
+    n = (np.arange(k) % 5).astype(np.int64)
+    wl = wi.Workload("wide", k, d, np.arange(k + 1, dtype=np.int64) * 4, n, 0.01, 0, 0.1, HINGE, 2, y, X=X)
+    assert_parity(P, wl)
+
+
+# ---- segmented runs and periodic averaging ----------------------------------------------------------------
+@pytest.mark.parametrize("variant", [1, 2, 3])
+def test_continue_equals_one_run(P, variant):
+    wl = wi.config1(k=3, d=64, m=128, n_steps=(203, 101, 50)).to("cuda")
+    wl.sched = 1  # the step number matters for eta_n, so a wrong restart shows
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("dense_variant", variant)
+        ctx.run_workload(wl)
+        full = ctx.get_models().cpu().numpy()
+        cuts = [np.array([50, 50, 50]), np.array([1, 1, 0]), np.array([152, 50, 0])]
+        ctx.run(wl.X, wl.y, wl.shard_off, cuts[0], wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        for c in cuts[1:]:
+            ctx.continue_(wl.X, wl.y, wl.shard_off, c)
+        seg = ctx.get_models().cpu().numpy()
+        wts, _ = ctx.get_weights()
+        ctx.check()
+    np.testing.assert_array_equal(seg, full)  # same arithmetic in the same order
+    owts, _, _ = oracle.weights(wl.n_steps, wl.eta0, wl.sched, wl.lam)
+    np.testing.assert_allclose(wts, owts, rtol=1e-12)
+
+
+def test_periodic_weighted_averaging(P):
+    # average every `span` fastest-node steps, then continue from the average on every node
+    wl = wi.config2(k=4, d=128, m=64, base_steps=120)
+    span_steps = [np.array([40, 20, 10, 40]), np.array([40, 20, 10, 40]), np.array([40, 20, 10, 40])]
+    dev = wl.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.run(dev.X, dev.y, wl.shard_off, span_steps[0], wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        for seg in span_steps[1:]:
+            ctx.set_models(ctx.combine())
+            ctx.continue_(dev.X, dev.y, wl.shard_off, seg)
+        v = ctx.combine().cpu().numpy()
+        ctx.check()
+    # oracle: same schedule; weights of each round come from that round's step counts
+    W = oracle.run_dense(wl.X, wl.y, wl.shard_off, span_steps[0], wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    done = span_steps[0].copy()
+    for seg in span_steps[1:]:
+        wts, _, _ = oracle.weights(done, wl.eta0, wl.sched, wl.lam)
+        vv = oracle.combine(W, wts)
+        # steps continue from each node's own count: run node by node with its own step_begin
+        Wn = np.zeros_like(W)
+        for j in range(wl.k):
+            only = np.zeros(wl.k, dtype=np.int64)
+            only[j] = seg[j]
+            Wn[j] = oracle.run_dense(wl.X, wl.y, wl.shard_off, only, wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed,
+                                     step_begin=int(done[j]), W_resume=np.tile(vv.astype(np.float32).astype(np.float64), (wl.k, 1)))[j]
+        W = Wn
+        done = done + seg
+    wts, _, _ = oracle.weights(done, wl.eta0, wl.sched, wl.lam)
+    assert rel_l2(v, oracle.combine(W, wts)) <= 1e-4
+
+
+# ---- evaluation measures ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_objective_and_error_rate(P, loss, bf16):
+    wl = wi.config1(k=2, d=64, m=333, n_steps=(10, 10))
+    X = wl.X.to(torch.bfloat16) if bf16 else wl.X
+    w = (torch.randn(64, generator=torch.Generator().manual_seed(4)) / 8)
+    with P.Context(2, 64) as ctx:
+        out = ctx.objective(X.cuda(), wl.y.cuda(), w.cuda(), 0.01, loss).cpu().numpy()
+        ctx.check()
+    obj, err = oracle.objective_dense(X, wl.y, w.numpy().astype(np.float64), 0.01, loss)
+    assert out[0] == pytest.approx(obj, rel=1e-5)
+    assert abs(out[1] - err) <= 2.0 / 666  # a margin within fp32 rounding of 0 may flip
+
+
+# ---- host-buffer entry point --------------------------------------------------------------------------------
+def test_solve_host_equals_device_path(P):
+    wl = wi.config2(k=5, d=256, m=128, base_steps=200)
+    wl.w0 = torch.full((256,), 0.5)
+    v_dev, _, _, _ = gpu_solve(P, wl)
+    with P.Context(wl.k, wl.d) as ctx:
+        out = ctx.solve_host(wl.X.pin_memory(), wl.y.pin_memory(), wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam,
+                             wl.loss, wl.seed, w0=wl.w0)
+        again = ctx.solve_host(wl.X, wl.y, wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed,
+                               w0=wl.w0)  # pageable source, buffers reused
+        ctx.check()
+    np.testing.assert_array_equal(out.numpy(), v_dev)
+    np.testing.assert_array_equal(again.numpy(), v_dev)
+
+
+# ---- sparse path --------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("prefetch", [2, 4, 8])
+def test_csr_losses_and_prefetch_depths(P, loss, prefetch):
+    wl = wi.config4(k=5, d=4096, m=300, base_steps=700, mean_nnz=30.0)
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.eta0 = 0.05
+    wl.w0 = torch.full((4096,), 0.01)
+    assert_parity(P, wl, {"prefetch": prefetch})
+
+
+def test_csr_long_rows_and_strong_regulariser(P):
+    # rows with up to 128 nonzeros (beyond the 64 kept in registers); eta*lambda large enough that the
+    # scale factor is folded back into the model several times
+    wl = wi.config4(k=3, d=512, m=64, base_steps=400, mean_nnz=90.0, max_nnz=128)
+    wl.sched, wl.eta0, wl.lam = 0, 0.5, 0.5  # (1 - 0.25)^400 ~ 1e-50
+    wl.w0 = torch.full((512,), 1.0)
+    assert_parity(P, wl)
+
+
+def test_csr_equals_dense_kernels_on_densified_rows(P):
+    wl = wi.config4(k=4, d=1024, m=128, base_steps=300, mean_nnz=20.0)
+    wl.loss = LOGISTIC
+    v_s, W_s, _, _ = gpu_solve(P, wl)
+    v_d, W_d, _, _ = gpu_solve(P, wi.densify(wl))
+    assert rel_l2(v_s, v_d) <= 1e-4
+
+
+# ---- argument checking ----------------------------------------------------------------------------------------
+def test_errors_are_reported_not_thrown_from_c(P):
+    wl = wi.config1(k=2, d=64, m=16, n_steps=(5, 5)).to("cuda")
+    with P.Context(2, 64) as ctx:
+        with pytest.raises(P.WpsgdError) as e:
+            ctx.combine()
+        assert e.value.status_name == "STATE"
+        with pytest.raises(P.WpsgdError) as e:
+            ctx.get_models()
+        assert e.value.status_name == "STATE"
+        bad = [dict(n_steps=np.array([5, -1])), dict(shard_off=np.array([0, 16, 8])), dict(eta0=float("nan")),
+               dict(lam=-1.0), dict(eta0=10.0, lam=0.2), dict(loss=9), dict(sched=5),
+               dict(shard_off=np.array([0, 0, 32]), n_steps=np.array([3, 3]))]
+        for kw in bad:
+            args = dict(shard_off=wl.shard_off, n_steps=wl.n_steps, eta0=wl.eta0, sched=wl.sched, lam=wl.lam,
+                        loss=wl.loss)
+            args.update(kw)
+            with pytest.raises(P.WpsgdError) as e:
+                ctx.run(wl.X, wl.y, args["shard_off"], args["n_steps"], args["eta0"], args["sched"], args["lam"],
+                        args["loss"], 0)
+            assert e.value.status_name == "INVALID_ARG", kw
+        with pytest.raises(P.WpsgdError):
+            ctx.set_option("no_such_option", 1)
+        with pytest.raises(P.WpsgdError):
+            ctx.sample_indices(0, 0, 0, 0, 4)
+        ctx.run_workload(wl)  # the context is still usable afterwards
+        ctx.combine()
+        ctx.check()
+        assert ctx.launch_count() >= 3
