@@ -164,6 +164,34 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, con
                               float lambda, wpsgd_loss loss, uint64_t seed, const float* w0, double r,
                               float* v_out);
 
+/* An entry point for callers that must not allocate device memory. (The paper has no counterpart:
+ * this is a convenience of the library.) It does what wpsgd_run followed by wpsgd_combine does on
+ * dense rows, but takes no context and calls no cudaMalloc / cudaFree or any other allocating
+ * routine: the model matrix, the sample stream and the small tables that a context would own live in
+ * one array built into the library (about 5.1 MiB of device memory on every GPU that loads it, held
+ * until the process exits). Meant for code that runs where allocation is forbidden or would stall:
+ * inside another framework's memory pool that has reserved the whole device, in a latency-critical
+ * loop that cannot afford cudaMalloc's device-wide synchronisation, or in a process whose memory
+ * budget is fixed at start-up.
+ *   device, cuda_stream   where to run; the work is enqueued on the stream and the call returns.
+ *   X, y, w0, v_out       DEVICE buffers of the caller, as in wpsgd_run / wpsgd_combine.
+ *   shard_off, n_steps    HOST [k+1] / [k], as in wpsgd_run.
+ * Limits (WPSGD_ERR_UNSUPPORTED with a message naming the limit when exceeded): k <=
+ * WPSGD_STATIC_MAX_NODES, k * d <= WPSGD_STATIC_MAX_MODEL_ELEMS, sum of n_steps <=
+ * WPSGD_STATIC_MAX_STEPS. Other argument errors as wpsgd_run.
+ * The first call on a device looks up the array's device address (once per device); make that
+ * first call before starting any stream capture. All calls on a device share the one array, which
+ * still holds what the previous call left there; each call rewrites what it uses and clears its
+ * status word, so calls in sequence on one stream are independent, but two calls whose GPU work
+ * overlaps (different streams, or different host threads) race on it and give wrong results. */
+#define WPSGD_STATIC_MAX_NODES 1024
+#define WPSGD_STATIC_MAX_MODEL_ELEMS (1 << 18)
+#define WPSGD_STATIC_MAX_STEPS (1 << 20)
+wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wpsgd_xtype xt, int64_t ld_elems,
+                                const float* y, const int64_t* shard_off, const int64_t* n_steps, int32_t k,
+                                int64_t d, float eta0, wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed,
+                                const float* w0, double r, float* v_out);
+
 /* Wait for the stream and read the device status word. WPSGD_OK, WPSGD_ERR_TIMEOUT (a bounded wait
  * gave up), or WPSGD_ERR_CUDA (a launch or copy failed, or a kernel's own bounds check fired). */
 wpsgd_status wpsgd_check(wpsgd_ctx* ctx);

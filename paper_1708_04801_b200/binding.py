@@ -16,7 +16,7 @@ _STATUS = {0: "OK", 1: "INVALID_ARG", 2: "ALLOC", 3: "CUDA", 4: "STATE", 5: "UNS
 EXPORTED_SYMBOLS = [
     "wpsgd_create", "wpsgd_destroy", "wpsgd_set_option", "wpsgd_set_node_ids", "wpsgd_run", "wpsgd_continue", "wpsgd_run_csr",
     "wpsgd_combine", "wpsgd_combine_weighted", "wpsgd_last_chain_ms", "wpsgd_get_models", "wpsgd_set_models", "wpsgd_get_weights", "wpsgd_weights",
-    "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_solve_host", "wpsgd_check", "wpsgd_launch_count",
+    "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_solve_host", "wpsgd_solve_static", "wpsgd_check", "wpsgd_launch_count",
     "wpsgd_last_error",
 ]
 
@@ -65,6 +65,7 @@ def load_library() -> ctypes.CDLL:
     lib.wpsgd_sample_indices.argtypes = [vp, u64, i32, i64, i64, i64, vp]
     lib.wpsgd_objective.argtypes = [vp, vp, ci, i64, vp, i64, vp, f32, ci, vp]
     lib.wpsgd_solve_host.argtypes = [vp, vp, ci, vp, vp, vp, f32, ci, f32, ci, u64, vp, f64, vp]
+    lib.wpsgd_solve_static.argtypes = [ci, vp, vp, ci, i64, vp, vp, vp, i32, i64, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_check.argtypes = [vp]
     lib.wpsgd_launch_count.argtypes = [vp]
     lib.wpsgd_launch_count.restype = i64
@@ -103,6 +104,35 @@ def _xtype(X) -> int:
     if X.dtype == torch.bfloat16:
         return X_BF16
     raise TypeError(f"features must be float32 or bfloat16, got {X.dtype}")
+
+
+def solve_static(X, y, shard_off, n_steps, eta0, sched, lam, loss, seed, w0=None, r: float = 0.0, out=None,
+                 stream=None):
+    """wpsgd_solve_static: chains plus combination on dense device tensors without a context and without
+    any device allocation by the library (its working memory is an array built into the library).
+    For callers that may not allocate; sizes are limited (see include/wpsgd.h). `out` should be given by
+    such callers; when it is None this wrapper allocates it with torch for convenience."""
+    import torch
+
+    lib = load_library()
+    if not X.is_cuda or X.dim() != 2 or X.stride(1) != 1:
+        raise TypeError("X must be a 2-D row-major CUDA tensor")
+    dev = X.device.index
+    so, ns = _host_i64(shard_off), _host_i64(n_steps)
+    k, d = ns.shape[0], X.shape[1]
+    if so.shape[0] != k + 1:
+        raise ValueError("shard_off must have k+1 entries")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=X.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev)
+    st = lib.wpsgd_solve_static(dev, ctypes.c_void_p(stream.cuda_stream), ctypes.c_void_p(X.data_ptr()), _xtype(X),
+                                X.stride(0), ctypes.c_void_p(y.data_ptr()), so.ctypes.data, ns.ctypes.data, k, d, eta0,
+                                sched, lam, loss, seed, ctypes.c_void_p(w0.data_ptr()) if w0 is not None else None, r,
+                                ctypes.c_void_p(out.data_ptr()))
+    if st:
+        raise WpsgdError(st, "wpsgd_solve_static", lib.wpsgd_last_error(None).decode())
+    return out
 
 
 class Context:

@@ -353,6 +353,56 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
 
 }  // namespace
 
+// ---- built-in scratch of the entry point that allocates nothing ----------------------------------------
+// Layout inside one file-scope device array (every section 256-byte aligned). The array exists once per
+// GPU that loads this library and lives until the process exits.
+namespace {
+constexpr size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+struct StaticLayout {
+  size_t W = 0;
+  size_t idx = align256(W + sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS);
+  size_t shard_off = align256(idx + sizeof(uint32_t) * (size_t)WPSGD_STATIC_MAX_STEPS);
+  size_t steps = align256(shard_off + sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
+  size_t first = align256(steps + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
+  size_t idx_off = align256(first + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
+  size_t rows = align256(idx_off + sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
+  size_t order = align256(rows + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
+  size_t ids = align256(order + sizeof(int) * WPSGD_STATIC_MAX_NODES);
+  size_t weights = align256(ids + sizeof(int) * WPSGD_STATIC_MAX_NODES);
+  size_t scale = align256(weights + sizeof(double) * WPSGD_STATIC_MAX_NODES);
+  size_t status = align256(scale + sizeof(double) * WPSGD_STATIC_MAX_NODES);
+  size_t total = align256(status + sizeof(DevStatus));
+};
+constexpr size_t kStaticBytes = align256(sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS) +
+                                align256(sizeof(uint32_t) * (size_t)WPSGD_STATIC_MAX_STEPS) +
+                                11 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
+constexpr int kStaticMaxDevices = 64;
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+namespace {
+// In host code the name g_static_scratch is only a handle of the symbol, not a device address; the address
+// a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device current.
+unsigned char* g_static_base[kStaticMaxDevices] = {nullptr};
+
+wpsgd_status static_scratch_base(int device, unsigned char** out) {
+  static_assert(sizeof(DevStatus) <= 256, "status word must fit its section");
+  if (StaticLayout().total > kStaticBytes) return fail(nullptr, WPSGD_ERR_STATE, "built-in scratch layout exceeds the array");
+  if (!g_static_base[device]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p) {
+      cudaGetLastError();
+      return fail(nullptr, WPSGD_ERR_CUDA, std::string("cudaGetSymbolAddress(built-in scratch): ") + cudaGetErrorString(e));
+    }
+    g_static_base[device] = (unsigned char*)p;
+  }
+  *out = g_static_base[device];
+  return WPSGD_OK;
+}
+}  // namespace
+
 extern "C" {
 
 wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, wpsgd_ctx** out) {
@@ -667,6 +717,78 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, const
   CU_TRY(c, cudaMemcpyAsync(v_out, c->st_v, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
   CU_TRY(c, cudaStreamSynchronize(c->stream));
   return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wpsgd_xtype xt, int64_t ld_elems,
+                                const float* y, const int64_t* shard_off, const int64_t* n_steps, int32_t k, int64_t d,
+                                float eta0, wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed,
+                                const float* w0, double r, float* v_out) {
+  if (k < 1 || d < 1) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "solve_static: k and d must be >= 1");
+  if (!shard_off || !n_steps || !v_out) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "solve_static: shard_off, n_steps or v_out is NULL");
+  char msg[200];
+  if (k > WPSGD_STATIC_MAX_NODES) {
+    snprintf(msg, sizeof(msg), "solve_static: k = %d exceeds the built-in maximum of %d nodes", (int)k, WPSGD_STATIC_MAX_NODES);
+    return fail(nullptr, WPSGD_ERR_UNSUPPORTED, msg);
+  }
+  if ((long long)k * (long long)d > WPSGD_STATIC_MAX_MODEL_ELEMS) {
+    snprintf(msg, sizeof(msg), "solve_static: k * d = %lld exceeds the built-in maximum of %lld model elements",
+             (long long)k * (long long)d, (long long)WPSGD_STATIC_MAX_MODEL_ELEMS);
+    return fail(nullptr, WPSGD_ERR_UNSUPPORTED, msg);
+  }
+  long long total = 0;
+  for (int j = 0; j < k; ++j) {
+    if (n_steps[j] < 0) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "solve_static: negative step count");
+    total += n_steps[j];
+    if (total > WPSGD_STATIC_MAX_STEPS) {
+      snprintf(msg, sizeof(msg), "solve_static: the step counts add up to more than the built-in maximum of %lld",
+               (long long)WPSGD_STATIC_MAX_STEPS);
+      return fail(nullptr, WPSGD_ERR_UNSUPPORTED, msg);
+    }
+  }
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    return fail(nullptr, WPSGD_ERR_CUDA, "no CUDA device available");
+  }
+  if (device < 0 || device >= ndev || device >= kStaticMaxDevices)
+    return fail(nullptr, WPSGD_ERR_INVALID_ARG, "solve_static: device index out of range");
+  DeviceGuard guard(device);
+  unsigned char* base = nullptr;
+  wpsgd_status s = static_scratch_base(device, &base);
+  if (s != WPSGD_OK) return s;
+
+  // A context on the host stack whose device pointers all lie inside the built-in array. It is never
+  // handed to wpsgd_destroy: nothing in it was allocated, so nothing is freed.
+  wpsgd_ctx c;
+  c.device = device;
+  c.stream = (cudaStream_t)cuda_stream;
+  c.k = k;
+  c.d = d;
+  c.steps_done.assign(k, 0);
+  c.node_ids.resize(k);
+  std::iota(c.node_ids.begin(), c.node_ids.end(), 0);
+  const StaticLayout L;
+  c.W = (float*)(base + L.W);
+  c.idx = (uint32_t*)(base + L.idx);
+  c.idx_cap = (size_t)WPSGD_STATIC_MAX_STEPS;  // so that the stream buffer is never regrown
+  c.t_shard_off = (long long*)(base + L.shard_off);
+  c.t_steps = (long long*)(base + L.steps);
+  c.t_first = (long long*)(base + L.first);
+  c.t_idx_off = (long long*)(base + L.idx_off);
+  c.t_rows = (long long*)(base + L.rows);
+  c.t_order = (int*)(base + L.order);
+  c.t_ids = (int*)(base + L.ids);
+  c.t_weights = (double*)(base + L.weights);
+  c.scale = (double*)(base + L.scale);
+  c.status = (DevStatus*)(base + L.status);
+  // the array keeps what the previous call left: the status word is the one thing that must start at zero
+  // (models, tables and the sample stream are fully rewritten for the sizes of this call)
+  cudaError_t e = cudaMemsetAsync(c.status, 0, sizeof(DevStatus), c.stream);
+  if (e != cudaSuccess) return fail(nullptr, WPSGD_ERR_CUDA, std::string("solve_static: cudaMemsetAsync: ") + cudaGetErrorString(e));
+  s = wpsgd_run(&c, X, xt, ld_elems, y, shard_off, n_steps, eta0, sched, lambda, loss, seed, w0);
+  if (s == WPSGD_OK) s = wpsgd_combine(&c, r, v_out);
+  if (s != WPSGD_OK) g_err = "solve_static: " + c.err;
+  return s;
 }
 
 wpsgd_status wpsgd_check(wpsgd_ctx* c) {
