@@ -10,6 +10,7 @@
 #include <string>
 #include <vector>
 
+#include "chain_block.cuh"
 #include "chain_csr.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
@@ -32,6 +33,7 @@ struct wpsgd_ctx {
   long long* t_first = nullptr;      // [k]
   long long* t_idx_off = nullptr;    // [k+1]
   long long* t_rows = nullptr;       // [k]
+  long long* t_count = nullptr;      // [k] entries of the sample stream per node (steps rounded up to 8)
   int* t_order = nullptr;            // [k]
   int* t_ids = nullptr;              // [k] node numbers entering the sample stream
   double* t_weights = nullptr;       // [k]
@@ -55,6 +57,7 @@ struct wpsgd_ctx {
   int sched = 0, loss = 0;
   uint64_t seed = 0;
   // options
+  int opt_stages = 0;
   int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_block_rows = 0, opt_cluster = 0, opt_sparse_threads = 32;
   long long opt_spin_limit = 1ll << 22;
   int opt_timing = 0;
@@ -177,7 +180,7 @@ int grid_for(long long work_items, int block, int cap = 148 * 16) {
 
 // ---- common part of run / continue: tables, sample stream ---------------------------------------------
 struct Plan {
-  std::vector<long long> off, steps, first, idx_off, rows;
+  std::vector<long long> off, steps, first, idx_off, rows, count;
   std::vector<int> order;
   long long total = 0;
 };
@@ -192,6 +195,7 @@ wpsgd_status make_plan(wpsgd_ctx* c, const long long* shard_off, const long long
   pl->first = first;
   pl->idx_off.assign(k + 1, 0);
   pl->rows.assign(k, 0);
+  pl->count.assign(k, 0);
   for (int j = 0; j < k; ++j) {
     const long long m = shard_off[j + 1] - shard_off[j];
     if (m < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off is not non-decreasing");
@@ -199,7 +203,10 @@ wpsgd_status make_plan(wpsgd_ctx* c, const long long* shard_off, const long long
     if (n_steps[j] > 0 && m < 1) return fail(c, WPSGD_ERR_INVALID_ARG, "a node with steps has an empty shard");
     if (m > 0xFFFFFFFFll) return fail(c, WPSGD_ERR_INVALID_ARG, "a shard has 2^32 rows or more");
     pl->rows[j] = m;
-    pl->idx_off[j + 1] = pl->idx_off[j] + n_steps[j];
+    // the stream of a node is produced up to the next multiple of 8 steps (the draws simply continue), so
+    // that kernels that take samples in groups always read valid rows
+    pl->count[j] = (n_steps[j] + 7) / 8 * 8;
+    pl->idx_off[j + 1] = pl->idx_off[j] + pl->count[j];
   }
   pl->total = pl->idx_off[k];
   pl->order.resize(k);
@@ -218,12 +225,13 @@ wpsgd_status upload_plan_and_stream(wpsgd_ctx* c, const Plan& pl) {
   CU_TRY(c, cudaMemcpyAsync(c->t_first, pl.first.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
   CU_TRY(c, cudaMemcpyAsync(c->t_idx_off, pl.idx_off.data(), (k + 1) * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
   CU_TRY(c, cudaMemcpyAsync(c->t_rows, pl.rows.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+  CU_TRY(c, cudaMemcpyAsync(c->t_count, pl.count.data(), k * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
   CU_TRY(c, cudaMemcpyAsync(c->t_order, pl.order.data(), k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CU_TRY(c, cudaMemcpyAsync(c->t_ids, c->node_ids.data(), k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   if (pl.total > 0) {
     const long long longest = *std::max_element(pl.steps.begin(), pl.steps.end());
     dim3 grid((unsigned)grid_for((longest + 3) / 4 + 1, 256, 1024), (unsigned)std::min(k, 65535));
-    index_stream_kernel<<<grid, 256, 0, c->stream>>>(c->seed, k, c->t_idx_off, c->t_first, c->t_steps, c->t_rows, c->t_ids, c->idx);
+    index_stream_kernel<<<grid, 256, 0, c->stream>>>(c->seed, k, c->t_idx_off, c->t_first, c->t_count, c->t_rows, c->t_ids, c->idx);
     CU_TRY(c, cudaGetLastError());
     c->launches++;
   }
@@ -280,6 +288,59 @@ wpsgd_status launch_reg_pf(wpsgd_ctx* c, const ChainParams& p, bool bpn, int thr
   }
 }
 
+// ---- blocked chain kernel: shapes it takes, ring depth, launch ------------------------------------------------
+constexpr size_t kSmemBudget = 220 * 1024;
+
+template <typename XT>
+bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* R_out, int* stages_out) {
+  constexpr int V = XVec<XT>::V;
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;  // keeps a^-8 harmless in fp32
+  const long long chunks = c->d / V;
+  const int math_threads = (int)std::min<long long>(32 * BLK_MAX_MATH_WARPS, (chunks + 31) / 32 * 32);
+  int R = (int)((chunks + math_threads - 1) / math_threads);
+  if (R > 4) return false;
+  if (R == 3) R = 4;
+  const size_t row_bytes = (size_t)c->d * sizeof(XT);
+  int stages = c->opt_stages > 0 ? c->opt_stages : 4;
+  while (stages >= 2 && BlockSmem(stages, row_bytes, math_threads / 32).total > kSmemBudget) --stages;
+  if (stages < 2) return false;
+  *threads_out = math_threads + 32;
+  *R_out = R;
+  *stages_out = stages;
+  return true;
+}
+
+template <typename XT, int R>
+wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, size_t smem) {
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<c->k, threads, smem, c->stream>>>(bp);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC>);
+    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED>);
+  }
+}
+
+template <typename XT>
+wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R, int stages) {
+  BlockParams bp;
+  bp.c = p;
+  bp.stages = stages;
+  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT), threads / 32 - 1).total;
+  switch (R) {
+    case 1: return launch_block_r<XT, 1>(c, bp, threads, smem);
+    case 2: return launch_block_r<XT, 2>(c, bp, threads, smem);
+    default: return launch_block_r<XT, 4>(c, bp, threads, smem);
+  }
+}
+
 template <typename XT>
 wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   constexpr int V = XVec<XT>::V;
@@ -288,9 +349,20 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                        ((uintptr_t)c->W % 16 == 0);
   const long long chunks = d / V;
   int variant = c->opt_variant;
+  int bthreads = 0, bR = 0, bstages = 0;
+  const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
   if (variant == 0) {
-    if (!aligned || chunks > 512 * 4) variant = 1;
-    else variant = (chunks <= 64) ? 3 : 2;
+    if (!aligned) variant = 1;
+    else if (chunks <= 64) variant = 3;
+    else if (block_ok) variant = 4;
+    else variant = (chunks > 512 * 4) ? 1 : 2;
+  }
+  if (variant == 4) {
+    if (!block_ok)
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "blocked kernel needs 16-byte aligned rows, a constant step size with eta*lambda <= 0.25, and d small "
+                  "enough for two 8-row blocks in shared memory");
+    return launch_block<XT>(c, p, bthreads, bR, bstages);
   }
   if ((variant == 2 || variant == 3) && !aligned)
     return fail(c, WPSGD_ERR_UNSUPPORTED, "register kernels need 16-byte aligned rows and d a multiple of 16 bytes");
@@ -361,12 +433,13 @@ constexpr size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 struct StaticLayout {
   size_t W = 0;
   size_t idx = align256(W + sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS);
-  size_t shard_off = align256(idx + sizeof(uint32_t) * (size_t)WPSGD_STATIC_MAX_STEPS);
+  size_t shard_off = align256(idx + sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES));
   size_t steps = align256(shard_off + sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
   size_t first = align256(steps + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t idx_off = align256(first + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t rows = align256(idx_off + sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
-  size_t order = align256(rows + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
+  size_t count = align256(rows + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
+  size_t order = align256(count + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t ids = align256(order + sizeof(int) * WPSGD_STATIC_MAX_NODES);
   size_t weights = align256(ids + sizeof(int) * WPSGD_STATIC_MAX_NODES);
   size_t scale = align256(weights + sizeof(double) * WPSGD_STATIC_MAX_NODES);
@@ -374,8 +447,8 @@ struct StaticLayout {
   size_t total = align256(status + sizeof(DevStatus));
 };
 constexpr size_t kStaticBytes = align256(sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS) +
-                                align256(sizeof(uint32_t) * (size_t)WPSGD_STATIC_MAX_STEPS) +
-                                11 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
+                                align256(sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES)) +
+                                12 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
 constexpr int kStaticMaxDevices = 64;
 }  // namespace
 
@@ -441,6 +514,7 @@ wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, w
   ALLOC(c->t_first, (size_t)k * sizeof(long long));
   ALLOC(c->t_idx_off, (size_t)(k + 1) * sizeof(long long));
   ALLOC(c->t_rows, (size_t)k * sizeof(long long));
+  ALLOC(c->t_count, (size_t)k * sizeof(long long));
   ALLOC(c->t_order, (size_t)k * sizeof(int));
   ALLOC(c->t_ids, (size_t)k * sizeof(int));
   ALLOC(c->t_weights, (size_t)k * sizeof(double));
@@ -455,7 +529,7 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* c) {
   if (!c) return WPSGD_OK;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  void* ptrs[] = {c->W, c->scale, c->t_shard_off, c->t_steps, c->t_first, c->t_idx_off, c->t_rows, c->t_order,
+  void* ptrs[] = {c->W, c->scale, c->t_shard_off, c->t_steps, c->t_first, c->t_idx_off, c->t_rows, c->t_count, c->t_order,
                   c->t_ids, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0};
   for (void* p : ptrs)
     if (p) cudaFree(p);
@@ -487,6 +561,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "sparse_threads") {
     if (value != 32) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_threads must be 32");
     c->opt_sparse_threads = (int)value;
+  } else if (n == "stages") {
+    if (value < 0 || value == 1 || value > 8) return fail(c, WPSGD_ERR_INVALID_ARG, "stages must be 0 or 2..8");
+    c->opt_stages = (int)value;
   } else if (n == "timing") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "timing must be 0 or 1");
     c->opt_timing = (int)value;
@@ -770,12 +847,13 @@ wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wp
   const StaticLayout L;
   c.W = (float*)(base + L.W);
   c.idx = (uint32_t*)(base + L.idx);
-  c.idx_cap = (size_t)WPSGD_STATIC_MAX_STEPS;  // so that the stream buffer is never regrown
+  c.idx_cap = (size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES;  // never regrown: padding included
   c.t_shard_off = (long long*)(base + L.shard_off);
   c.t_steps = (long long*)(base + L.steps);
   c.t_first = (long long*)(base + L.first);
   c.t_idx_off = (long long*)(base + L.idx_off);
   c.t_rows = (long long*)(base + L.rows);
+  c.t_count = (long long*)(base + L.count);
   c.t_order = (int*)(base + L.order);
   c.t_ids = (int*)(base + L.ids);
   c.t_weights = (double*)(base + L.weights);

@@ -76,7 +76,7 @@ def test_small_workloads_default_kernels(P, cfg):
 
 # ---- every dense kernel variant ----------------------------------------------------------------------
 @pytest.mark.parametrize("variant,threads,prefetch", [(1, 0, 0), (2, 0, 2), (2, 0, 4), (2, 0, 8), (2, 128, 4), (2, 64, 8),
-                                                      (2, 32, 2), (3, 0, 2), (3, 0, 4), (3, 0, 8)])
+                                                      (2, 32, 2), (3, 0, 2), (3, 0, 4), (3, 0, 8), (4, 0, 0)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_dense_variants(P, variant, threads, prefetch, bf16):
     # d = 480: 120 fp32 / 60 bf16 16-byte chunks: ragged against 32-lane and 128-thread tiles
@@ -88,10 +88,15 @@ def test_dense_variants(P, variant, threads, prefetch, bf16):
 
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
 @pytest.mark.parametrize("sched", [0, 1])
-@pytest.mark.parametrize("variant", [1, 2, 3])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4])
 def test_losses_and_schedules(P, loss, sched, variant):
     wl = wi.config1(k=3, d=64, m=128, n_steps=(300, 150, 40))
     wl.loss, wl.sched = loss, sched
+    if variant == 4 and sched == 1:  # the blocked kernel is for the constant step size
+        with pytest.raises(P.WpsgdError) as e:
+            gpu_solve(P, wl, {"dense_variant": 4})
+        assert e.value.status_name == "UNSUPPORTED"
+        return
     wl.eta0 = 0.05 if sched else 0.01
     if loss == SQUARED:
         wl.y = (wl.y * 0.5 + 0.1).contiguous()
@@ -124,6 +129,40 @@ def test_generic_kernel_handles_unaligned_shapes(P):
 def test_large_d_falls_back_and_matches(P):
     wl = wi.config2(k=2, d=8200, m=16, base_steps=40)  # beyond the register kernels' reach
     assert_parity(P, wl)
+
+
+# ---- blocked kernel: block boundaries, ring depths, column tilings ----------------------------------------
+@pytest.mark.parametrize("n_steps", [(1, 7, 8), (9, 15, 16), (17, 0, 64), (333, 250, 3)])
+@pytest.mark.parametrize("stages", [2, 3, 4])
+def test_blocked_kernel_block_boundaries_and_ring_depths(P, n_steps, stages):
+    wl = wi.config2(k=3, d=1024, m=64, base_steps=8)
+    wl.n_steps = np.array(n_steps, dtype=np.int64)
+    wl.w0 = torch.full((1024,), 0.1)
+    assert_parity(P, wl, {"dense_variant": 4, "stages": stages})
+
+
+@pytest.mark.parametrize("d,bf16", [(64, False), (480, False), (1024, False), (2048, False), (3072, False), (64, True),
+                                     (1000, True), (4096, True), (6144, True)])
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+def test_blocked_kernel_column_tilings(P, d, bf16, loss):
+    wl = wi.config2(k=3, d=d, m=48, base_steps=210)
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    if bf16:
+        wl.X = wl.X.to(torch.bfloat16)
+    assert_parity(P, wl, {"dense_variant": 4})
+
+
+def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
+    wl = wi.config2(k=4, d=1024, m=64, base_steps=100).to("cuda")
+    with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
+        a.run_workload(wl)
+        b.set_option("dense_variant", 4)
+        b.run_workload(wl)
+        np.testing.assert_array_equal(a.get_models().cpu().numpy(), b.get_models().cpu().numpy())
+        a.check()
+        b.check()
 
 
 # ---- degenerate cases -----------------------------------------------------------------------------------
@@ -206,6 +245,23 @@ def test_combine_many_nodes_ragged_d(P):
 
 
 # ---- segmented runs and periodic averaging ----------------------------------------------------------------
+def test_continue_blocked_kernel(P):
+    # the blocked kernel groups samples by eight from wherever a segment starts, so a cut run agrees with the
+    # uncut one up to rounding order (not bit for bit)
+    wl_cpu = wi.config2(k=3, d=256, m=128, base_steps=203)
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("dense_variant", 4)
+        first = np.minimum(wl.n_steps, 37)
+        ctx.run(wl.X, wl.y, wl.shard_off, first, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        ctx.continue_(wl.X, wl.y, wl.shard_off, wl.n_steps - first)
+        seg = ctx.get_models().cpu().numpy()
+        ctx.check()
+    oW = oracle.run_dense(wl_cpu.X, wl_cpu.y, wl.shard_off, wl.n_steps, wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    for j in range(wl.k):
+        assert rel_l2(seg[j], oW[j]) <= 1e-4
+
+
 @pytest.mark.parametrize("variant", [1, 2, 3])
 def test_continue_equals_one_run(P, variant):
     wl = wi.config1(k=3, d=64, m=128, n_steps=(203, 101, 50)).to("cuda")
