@@ -55,14 +55,6 @@ __device__ __forceinline__ void cp_async_wait(int pending) {
   }
 }
 
-// dL/dz with the fast exponential and reciprocal units (relative error of a few 2^-22)
-template <int LOSS>
-__device__ __forceinline__ float loss_derivative_fast(float y, float z) {
-  if (LOSS == LOSS_HINGE) return (y * z < 1.0f) ? -y : 0.0f;
-  if (LOSS == LOSS_LOGISTIC) return __fdividef(-y, 1.0f + __expf(y * z));
-  return z - y;
-}
-
 // Quad q (4 consecutive columns) of a 16-byte chunk, widened to fp32.
 template <typename XT>
 __device__ __forceinline__ void widen_quad(const uint4& raw, int q, float (&f)[4]);
@@ -121,20 +113,20 @@ constexpr int BLK_MAX_MATH_WARPS = 8;
 
 // Shared-memory carve-up (bytes). Ring first (16-byte aligned), then the small arrays.
 struct BlockSmem {
-  size_t ring, ys, redG, redP, totG, gam, tab, total;
+  size_t ring, redG, redP, totG, gam, tab, total;
   __host__ __device__ BlockSmem(int stages, size_t row_bytes, int math_warps) {
     ring = 0;
-    ys = ring + (size_t)stages * BLK_B * row_bytes;
-    redG = ys + (size_t)stages * BLK_B * sizeof(float);
-    redP = redG + (size_t)math_warps * 32 * sizeof(float);
-    totG = redP + (size_t)math_warps * BLK_B * sizeof(float);
+    redG = ring + (size_t)stages * BLK_B * row_bytes;
+    (void)math_warps;  // the partial-sum arrays always have room for the maximum number of math warps
+    redP = redG + (size_t)BLK_MAX_MATH_WARPS * 32 * sizeof(float);
+    totG = redP + (size_t)BLK_MAX_MATH_WARPS * BLK_B * sizeof(float);
     gam = totG + 32 * sizeof(float);
     tab = gam + 16 * sizeof(float);
     total = tab + 3 * 16 * sizeof(float);
   }
 };
 
-template <typename XT, int R, int LOSS>
+template <typename XT, int R, int LOSS, bool OVERLAP>
 __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;   // columns per 16-byte chunk
   constexpr int QV = V / 4;        // quads per chunk
@@ -152,12 +144,11 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
   const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
   const BlockSmem L(S, row_bytes, math_warps);
   unsigned char* ring = smem + L.ring;
-  float* ys = (float*)(smem + L.ys);
-  float* redG = (float*)(smem + L.redG);
-  float* redP = (float*)(smem + L.redP);
-  float* totG = (float*)(smem + L.totG);
-  float* gam = (float*)(smem + L.gam);   // gamma_0..7, [8] = 1 - a^nv
-  float* tab = (float*)(smem + L.tab);   // [0..8] a^k, [16..24] eta / a^{k+1}, [32..40] 1 - a^k
+  float* redG = (float*)(smem + L.redG);   // [math warp][32] partial Gram entries
+  float* redP = (float*)(smem + L.redP);   // [math warp][8] partial p
+  float* totG = (float*)(smem + L.totG);   // [32] Gram entries summed over the math warps
+  float* gam = (float*)(smem + L.gam);     // gamma_0..7, [8] = 1 - a^nv
+  float* tab = (float*)(smem + L.tab);     // [0..8] a^k, [16..24] eta / a^{k+1}, [32..40] 1 - a^k
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes;
   const float* yshard = p.y + p.shard_off[j];
   const uint32_t* idx = p.idx + p.idx_off[j];  // padded to a multiple of B entries, all valid rows
@@ -174,45 +165,98 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
 
   if (warp == 0) {
     // =========================== serial warp ===========================================================
-    const int n = lane & (B - 1);  // sample of the block this lane stands for (lanes >= B mirror, unused)
-    // label prefetch: lane n < B copies y of sample n of blocks 0..S-1
-    for (int s = 0; s < S; ++s) {
-      if (lane < B && s < nb) cp_async4(&ys[s * B + lane], yshard + idx[(long long)s * B + lane]);
-      cp_async_commit();
-    }
+    // Every lane runs the whole B-step recurrence redundantly on its own copy of the block's scalars (no
+    // shuffle inside the dependent chain); lanes only differ in which partial sums they add up and in
+    // which gamma they store. Lane n & 7 looks after the label of sample n.
+    const int n = lane & (B - 1);
+    for (int i = lane; i < BLK_MAX_MATH_WARPS * 32; i += 32)  // unused partial-sum slots read as zero
+      if (i >= math_warps * 32) redG[i] = 0.0f;
+    for (int i = lane; i < BLK_MAX_MATH_WARPS * B; i += 32)
+      if (i >= math_warps * B) redP[i] = 0.0f;
+    // label pipeline in registers: label of block b+1 and sample id of block b+2 are in flight during block b
+    float y_nxt = 0.0f;
+    uint32_t id_nxt = 0u;
+    if (nb > 0) y_nxt = yshard[idx[n]];
+    if (nb > 1) id_nxt = idx[B + n];
     __syncthreads();  // tables visible (pairs with the math warps' first barrier)
-    const float apow_n = tab[n], cfac_n = tab[16 + n];
+    float apw[B], cfac[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+
     for (long long b = 0; b < nb; ++b) {
       const int nv = (int)((n_run - b * B) < (long long)B ? (n_run - b * B) : (long long)B);
-      // totals of G_b (partials were written by the math warps before the previous barrier 2)
-      float g_tot = 0.0f;
-      for (int w = 0; w < math_warps; ++w) g_tot += redG[w * 32 + lane];
-      totG[lane] = g_tot;
-      __syncwarp();
-      float gcol[B];  // gcol[m] = G[m][n] for m < n
-#pragma unroll
-      for (int m = 0; m < B; ++m) gcol[m] = (m < n) ? totG[n * (n - 1) / 2 + m] : 0.0f;
-      cp_async_wait(S - 1 < 3 ? S - 1 : 3);  // this lane's label of block b has landed
-      const float yn = ys[(int)(b % S) * B + n];
-      __syncthreads();  // barrier 1: p_b partials are in redP
-      float zacc = 0.0f;
-      for (int w = 0; w < math_warps; ++w) zacc += redP[w * B + n];
-      const float c_n = (n < nv) ? cfac_n : 0.0f;  // samples beyond the chain's end take no step
-      float g_own = 0.0f;
+      const float y_cur = y_nxt;
+      if (b + 1 < nb) y_nxt = yshard[id_nxt];
+      if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
+      const float a_nv = tab[nv], dl_nv = tab[32 + nv];
+      // per-sample constants with everything folded in that does not depend on the chain:
+      // t_n = sc_n (p_n - sum_m beta_m G_mn) is the argument of the loss derivative, beta_n = cf_n * f(t_n)
+      float yv[B], sc[B], cf[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) {
-        const float z = apow_n * zacc;
-        const float g = loss_derivative_fast<LOSS>(yn, z);
-        if (m == n) g_own = g;
-        const float beta_m = __shfl_sync(0xffffffffu, c_n * g, m);
-        zacc = fmaf(-beta_m, gcol[m], zacc);
+        yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+        if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
+          sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
+          cf[m] = -yv[m] * cfac[m];
+        } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
+          sc[m] = yv[m] * apw[m];
+          cf[m] = -yv[m] * cfac[m];
+        } else {  // g = t - y, t = a^n (...)
+          sc[m] = apw[m];
+          cf[m] = cfac[m];
+        }
+        if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
       }
-      // gamma_n = eta g_n a^{nv-1-n}; tab[16+k] = eta / a^{k+1}, so use eta0 * a^{nv-1-n} directly
-      if (lane < B) gam[lane] = (lane < nv) ? p.eta0 * g_own * tab[nv - 1 - lane] : 0.0f;
-      if (lane == B) gam[B] = tab[32 + nv];
+      float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
+      auto gather_gram = [&]() {
+        float gp[BLK_MAX_MATH_WARPS];
+#pragma unroll
+        for (int w = 0; w < BLK_MAX_MATH_WARPS; ++w) gp[w] = redG[w * 32 + lane];
+        totG[lane] = ((gp[0] + gp[1]) + (gp[2] + gp[3])) + ((gp[4] + gp[5]) + (gp[6] + gp[7]));
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < BLK_PAIRS / 4; ++i) {
+          const float4 q = ((const float4*)totG)[i];
+          Gs[4 * i] = q.x; Gs[4 * i + 1] = q.y; Gs[4 * i + 2] = q.z; Gs[4 * i + 3] = q.w;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+          for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] *= sc[n2];
+      };
+      if (OVERLAP) gather_gram();  // G_b was finished by the math warps during the previous block
+      __syncthreads();             // barrier 1: p_b partials (and, without overlap, G_b partials) are in place
+      if (!OVERLAP) gather_gram();
+      float pp[BLK_MAX_MATH_WARPS];
+#pragma unroll
+      for (int w = 0; w < BLK_MAX_MATH_WARPS; ++w) pp[w] = redP[w * B + n];
+      const float psum = ((pp[0] + pp[1]) + (pp[2] + pp[3])) + ((pp[4] + pp[5]) + (pp[6] + pp[7]));
+      float t[B], beta[B];
+#pragma unroll
+      for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        if (LOSS == LOSS_LOGISTIC) {
+          float e, r;
+          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t[m]));
+          asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+          beta[m] = cf[m] * r;
+        } else if (LOSS == LOSS_HINGE) {
+          beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+        } else {
+          beta[m] = cf[m] * (t[m] - yv[m]);
+        }
+#pragma unroll
+        for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+      }
+      // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}
+      float mine = dl_nv;
+#pragma unroll
+      for (int m = 0; m < B; ++m)
+        if (lane == m) mine = beta[m] * a_nv;
+      if (lane <= B) gam[lane] = mine;
       __syncthreads();  // barrier 2: gamma published
-      if (lane < B && b + S < nb) cp_async4(&ys[(int)(b % S) * B + lane], yshard + idx[(b + S) * B + lane]);
-      cp_async_commit();
     }
     return;
   }
@@ -236,11 +280,19 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     }
   }
 
-  // issue the copies of this thread's chunks of block blk into its ring stage
-  auto prefetch_block = [&](long long blk) {
+  // sample ids of a block: 8 consecutive entries, 32-byte aligned (every node's stream starts on a multiple of 8)
+  auto load_ids = [&](long long blk, uint4& lo, uint4& hi) {
     if (blk < nb) {
-      unsigned char* stage = ring + (size_t)(blk % S) * B * row_bytes;
-      const uint32_t* ib = idx + blk * B;
+      const uint4* q = (const uint4*)(idx + blk * B);
+      lo = __ldg(q);
+      hi = __ldg(q + 1);
+    }
+  };
+  // issue the copies of this thread's chunks of block blk into ring stage stg (one commit group per call)
+  auto prefetch_block = [&](long long blk, int stg, const uint4& i_lo, const uint4& i_hi) {
+    if (blk < nb) {
+      unsigned char* stage = ring + (size_t)stg * B * row_bytes;
+      const uint32_t ib[B] = {i_lo.x, i_lo.y, i_lo.z, i_lo.w, i_hi.x, i_hi.y, i_hi.z, i_hi.w};
 #pragma unroll
       for (int m = 0; m < B; ++m) {
         const char* row = shard + (size_t)ib[m] * ld_bytes;
@@ -251,94 +303,144 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     }
     cp_async_commit();
   };
-  // G partials of block blk -> redG (each warp its own 32 slots)
-  auto gram_block = [&](long long blk) {
-    float acc[32];
+  // this thread's chunks of the 8 rows of a landed block, shared memory -> registers (the only read of them)
+  auto load_raw = [&](int stg, uint4 (&raw)[R][B]) {
+    const unsigned char* stage = ring + (size_t)stg * B * row_bytes;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-    if (blk < nb) {
-      const unsigned char* stage = ring + (size_t)(blk % S) * B * row_bytes;
+    for (int r = 0; r < R; ++r)
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        if (!act[r]) continue;
-        uint4 raw[B];
+      for (int m = 0; m < B; ++m)
+        raw[r][m] = act[r] ? *(const uint4*)(stage + (size_t)m * row_bytes + ((size_t)r * TM + tm) * 16)
+                           : make_uint4(0u, 0u, 0u, 0u);
+  };
+  // Gram partials (and, when WITH_P, p partials against the current model) of the block held in raw
+  auto products = [&](const uint4 (&raw)[R][B], float (&acc)[32], float (&accp)[B], bool with_g, bool with_p) {
 #pragma unroll
-        for (int m = 0; m < B; ++m)
-          raw[m] = *(const uint4*)(stage + (size_t)m * row_bytes + ((size_t)r * TM + tm) * 16);
+    for (int r = 0; r < R; ++r) {
 #pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          float x[B][4];
+      for (int q = 0; q < QV; ++q) {
+        float x[B][4];
 #pragma unroll
-          for (int m = 0; m < B; ++m) widen_quad<XT>(raw[m], q, x[m]);
+        for (int m = 0; m < B; ++m) widen_quad<XT>(raw[r][m], q, x[m]);
+        if (with_g) {
 #pragma unroll
           for (int n2 = 1; n2 < B; ++n2)
 #pragma unroll
             for (int m = 0; m < n2; ++m)
 #pragma unroll
-              for (int e = 0; e < 4; ++e) acc[n2 * (n2 - 1) / 2 + m] = fmaf(x[m][e], x[n2][e], acc[n2 * (n2 - 1) / 2 + m]);
+              for (int e = 0; e < 4; ++e)
+                acc[n2 * (n2 - 1) / 2 + m] = fmaf(x[m][e], x[n2][e], acc[n2 * (n2 - 1) / 2 + m]);
+        }
+        if (with_p) {
+#pragma unroll
+          for (int m = 0; m < B; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) accp[m] = fmaf(w[r][q * 4 + e], x[m][e], accp[m]);
         }
       }
     }
+  };
+  auto publish_g = [&](float (&acc)[32]) {
     const float tot = warp_transpose_sum32(acc);
     redG[(warp - 1) * 32 + lane] = tot;
   };
-
-  for (int s = 0; s < S; ++s) prefetch_block(s);
-  cp_async_wait(S - 1 < 3 ? S - 1 : 3);  // block 0 has landed
-  gram_block(0);
-  __syncthreads();  // tables visible; G_0 partials visible to the serial warp
-
-  for (long long b = 0; b < nb; ++b) {
-    const unsigned char* stage = ring + (size_t)(b % S) * B * row_bytes;
-    // ---- p_b = X_b w ---------------------------------------------------------------------------------
-    float accp[B];
-#pragma unroll
-    for (int m = 0; m < B; ++m) accp[m] = 0.0f;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      if (!act[r]) continue;
-#pragma unroll
-      for (int m = 0; m < B; ++m) {
-        const uint4 raw = *(const uint4*)(stage + (size_t)m * row_bytes + ((size_t)r * TM + tm) * 16);
-#pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          float x[4];
-          widen_quad<XT>(raw, q, x);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) accp[m] = fmaf(w[r][q * 4 + e], x[e], accp[m]);
-        }
-      }
-    }
+  auto publish_p = [&](float (&accp)[B]) {
     const float ptot = warp_transpose_sum8(accp);
     if ((lane & 3) == 0) redP[(warp - 1) * B + (lane >> 2)] = ptot;
-    __syncthreads();  // barrier 1
-    // ---- G_{b+1}, off the serial path -----------------------------------------------------------------
-    cp_async_wait(S - 2 < 3 ? S - 2 : 3);  // block b+1 has landed
-    gram_block(b + 1);
-    __syncthreads();  // barrier 2: gamma_b is in gam
-    // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m -------------------------------------------------------
+  };
+  // w <- w - (1 - a^nv) w - sum_m gamma_m x_m with the rows held in raw
+  auto update = [&](const uint4 (&raw)[R][B]) {
     float gm[B];
 #pragma unroll
     for (int m = 0; m < B; ++m) gm[m] = gam[m];
     const float dl = gam[B];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (!act[r]) continue;
 #pragma unroll
       for (int v = 0; v < V; ++v) w[r][v] = fmaf(-dl, w[r][v], w[r][v]);
 #pragma unroll
-      for (int m = 0; m < B; ++m) {
-        const uint4 raw = *(const uint4*)(stage + (size_t)m * row_bytes + ((size_t)r * TM + tm) * 16);
+      for (int m = 0; m < B; ++m)
 #pragma unroll
         for (int q = 0; q < QV; ++q) {
           float x[4];
-          widen_quad<XT>(raw, q, x);
+          widen_quad<XT>(raw[r][m], q, x);
 #pragma unroll
           for (int e = 0; e < 4; ++e) w[r][q * 4 + e] = fmaf(-gm[m], x[e], w[r][q * 4 + e]);
         }
-      }
     }
-    prefetch_block(b + S);  // the stage of block b is free again
+  };
+
+  uint4 id_lo = make_uint4(0, 0, 0, 0), id_hi = make_uint4(0, 0, 0, 0);
+  for (int s = 0; s < S; ++s) {
+    load_ids(s, id_lo, id_hi);
+    prefetch_block(s, s, id_lo, id_hi);
+  }
+  load_ids(S, id_lo, id_hi);
+  float acc[32], accp[B];
+
+  if (OVERLAP) {
+    // Two register copies of row blocks: `cur` (block b: p_b, update) and `nxt` (block b+1: G_{b+1}).
+    uint4 cur[R][B], nxt[R][B];
+    cp_async_wait(S - 1 < 3 ? S - 1 : 3);  // block 0 has landed
+    load_raw(0, cur);
+    prefetch_block(S, 0, id_lo, id_hi);    // its stage is free again at once
+    load_ids(S + 1, id_lo, id_hi);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+    products(cur, acc, accp, true, false);
+    publish_g(acc);
+    __syncthreads();  // tables visible; G_0 partials visible to the serial warp
+    int st = (S > 1) ? 1 : 0;  // ring stage of block b+1
+    for (long long b = 0; b < nb; ++b) {
+#pragma unroll
+      for (int m = 0; m < B; ++m) accp[m] = 0.0f;
+      products(cur, acc, accp, false, true);  // p_b = X_b w
+      publish_p(accp);
+      __syncthreads();  // barrier 1
+      // G_{b+1}, off the serial path
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+      if (b + 1 < nb) {
+        // groups committed so far: S + 1 + b (blocks 0 .. S+b); block b+1 must be complete
+        cp_async_wait(S - 1 < 3 ? S - 1 : 3);
+        load_raw(st, nxt);
+        products(nxt, acc, accp, true, false);
+      }
+      prefetch_block(b + 1 + S, st, id_lo, id_hi);
+      load_ids(b + 2 + S, id_lo, id_hi);
+      publish_g(acc);
+      __syncthreads();  // barrier 2: gamma_b is in gam
+      update(cur);
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int m = 0; m < B; ++m) cur[r][m] = nxt[r][m];
+      st = (st + 1 == S) ? 0 : st + 1;
+    }
+  } else {
+    // One register copy: the block is read once, G_b and p_b are formed in the same pass over it, and the
+    // rows stay in registers across the serial phase for the update.
+    uint4 cur[R][B];
+    __syncthreads();  // tables visible
+    int st = 0;       // ring stage of block b
+    for (long long b = 0; b < nb; ++b) {
+      // groups committed so far: S + b (blocks 0 .. S+b-1); block b must be complete
+      cp_async_wait(S - 1 < 3 ? S - 1 : 3);
+      load_raw(st, cur);
+      prefetch_block(b + S, st, id_lo, id_hi);
+      load_ids(b + 1 + S, id_lo, id_hi);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+#pragma unroll
+      for (int m = 0; m < B; ++m) accp[m] = 0.0f;
+      products(cur, acc, accp, true, true);
+      publish_p(accp);
+      publish_g(acc);
+      __syncthreads();  // barrier 1
+      __syncthreads();  // barrier 2: gamma_b is in gam
+      update(cur);
+      st = (st + 1 == S) ? 0 : st + 1;
+    }
   }
   cp_async_wait(0);
 

@@ -299,8 +299,7 @@ bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* 
   const long long chunks = c->d / V;
   const int math_threads = (int)std::min<long long>(32 * BLK_MAX_MATH_WARPS, (chunks + 31) / 32 * 32);
   int R = (int)((chunks + math_threads - 1) / math_threads);
-  if (R > 4) return false;
-  if (R == 3) R = 4;
+  if (R > 2) return false;  // beyond two chunks per thread the rows of a block no longer fit in registers
   const size_t row_bytes = (size_t)c->d * sizeof(XT);
   int stages = c->opt_stages > 0 ? c->opt_stages : 4;
   while (stages >= 2 && BlockSmem(stages, row_bytes, math_threads / 32).total > kSmemBudget) --stages;
@@ -321,9 +320,11 @@ wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, si
     return WPSGD_OK;
   };
   switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC>);
-    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED>);
+    // one 16-byte chunk per thread: room for two register copies of a block, so the Gram products of the
+    // next block overlap the serial recurrence; more chunks: one copy, Gram and p in the same pass
+    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, R == 1>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, R == 1>);
+    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, R == 1>);
   }
 }
 
@@ -336,8 +337,7 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
   const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT), threads / 32 - 1).total;
   switch (R) {
     case 1: return launch_block_r<XT, 1>(c, bp, threads, smem);
-    case 2: return launch_block_r<XT, 2>(c, bp, threads, smem);
-    default: return launch_block_r<XT, 4>(c, bp, threads, smem);
+    default: return launch_block_r<XT, 2>(c, bp, threads, smem);
   }
 }
 
@@ -360,8 +360,7 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   if (variant == 4) {
     if (!block_ok)
       return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "blocked kernel needs 16-byte aligned rows, a constant step size with eta*lambda <= 0.25, and d small "
-                  "enough for two 8-row blocks in shared memory");
+                  "blocked kernel needs 16-byte aligned rows of at most 8 KiB, a constant step size and eta*lambda <= 0.25");
     return launch_block<XT>(c, p, bthreads, bR, bstages);
   }
   if ((variant == 2 || variant == 3) && !aligned)

@@ -141,8 +141,8 @@ def test_blocked_kernel_block_boundaries_and_ring_depths(P, n_steps, stages):
     assert_parity(P, wl, {"dense_variant": 4, "stages": stages})
 
 
-@pytest.mark.parametrize("d,bf16", [(64, False), (480, False), (1024, False), (2048, False), (3072, False), (64, True),
-                                     (1000, True), (4096, True), (6144, True)])
+@pytest.mark.parametrize("d,bf16", [(64, False), (480, False), (1024, False), (2048, False), (1536, False), (64, True),
+                                     (1000, True), (4096, True), (3008, True)])
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
 def test_blocked_kernel_column_tilings(P, d, bf16, loss):
     wl = wi.config2(k=3, d=d, m=48, base_steps=210)
