@@ -456,3 +456,239 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
 }
 
 }  // namespace wpsgd
+
+// ======================================================================================================
+// Small d: one warp per node, several nodes per CTA. The same blocked form, with no CTA-wide barrier at
+// all: the warp forms G_b and p_b in one pass over its 8 rows (each lane owns R 16-byte column chunks),
+// sums them over its lanes, every lane then runs the 8-step recurrence redundantly and applies the
+// update from registers. Rows arrive through a per-warp ring filled by the lanes' own asynchronous copies.
+// ======================================================================================================
+namespace wpsgd {
+
+constexpr int BLKW_WARPS = 4;  // nodes per CTA
+
+struct BlockWarpSmem {
+  size_t ring, scratch, tab, total;
+  __host__ __device__ BlockWarpSmem(int stages, size_t row_bytes) {
+    ring = 0;
+    scratch = ring + (size_t)BLKW_WARPS * stages * BLK_B * row_bytes;
+    tab = scratch + (size_t)BLKW_WARPS * 48 * sizeof(float);
+    total = tab + 3 * 16 * sizeof(float);
+  }
+};
+
+template <typename XT, int R, int LOSS>
+__global__ void __launch_bounds__(32 * BLKW_WARPS) chain_block_warp_kernel(const BlockParams bp) {
+  constexpr int V = XVec<XT>::V;
+  constexpr int QV = V / 4;
+  constexpr int B = BLK_B;
+  extern __shared__ __align__(16) unsigned char smem[];
+  const ChainParams& p = bp.c;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int S = bp.stages;
+  const long long d = p.d;
+  const size_t row_bytes = (size_t)d * sizeof(XT);
+  const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
+  const BlockWarpSmem L(S, row_bytes);
+  unsigned char* ring = smem + L.ring + (size_t)warp * S * B * row_bytes;
+  float* scratch = (float*)(smem + L.scratch) + warp * 48;  // [0..27] G entries, [32..39] p
+  float* tab = (float*)(smem + L.tab);
+
+  if (threadIdx.x <= B) {  // power tables in fp64, rounded once
+    const double a = 1.0 - bp.eta_lambda;
+    double pw = 1.0;
+    for (int k = 0; k < (int)threadIdx.x; ++k) pw *= a;
+    tab[threadIdx.x] = (float)pw;
+    tab[16 + threadIdx.x] = (float)((double)p.eta0 / (pw * a));
+    tab[32 + threadIdx.x] = (float)(1.0 - pw);
+  }
+  __syncthreads();  // the only CTA-wide barrier; every warp passes it exactly once
+  const int slot = (int)blockIdx.x * BLKW_WARPS + warp;
+  if (slot >= p.k) return;
+  const int j = p.order[slot];
+  const long long n_run = p.n_steps[j];
+  const long long nb = (n_run + B - 1) / B;
+  const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes;
+  const float* yshard = p.y + p.shard_off[j];
+  const uint32_t* idx = p.idx + p.idx_off[j];
+  const int n = lane & (B - 1);
+
+  float apw[B], cfac[B];
+#pragma unroll
+  for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+
+  bool act[R];
+  float w[R][V];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const long long c0 = ((long long)r * 32 + lane) * V;
+    act[r] = c0 < d;
+#pragma unroll
+    for (int v = 0; v < V; ++v) w[r][v] = 0.0f;
+    if (act[r]) {
+      const float* src = p.resume ? (p.W + (size_t)j * d + c0) : (p.w0 ? p.w0 + c0 : nullptr);
+      if (src) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) w[r][v] = src[v];
+      }
+    }
+  }
+
+  auto load_ids = [&](long long blk, uint4& lo, uint4& hi) {
+    if (blk < nb) {
+      const uint4* q = (const uint4*)(idx + blk * B);
+      lo = __ldg(q);
+      hi = __ldg(q + 1);
+    }
+  };
+  auto prefetch_block = [&](long long blk, int stg, const uint4& i_lo, const uint4& i_hi) {
+    if (blk < nb) {
+      unsigned char* stage = ring + (size_t)stg * B * row_bytes;
+      const uint32_t ib[B] = {i_lo.x, i_lo.y, i_lo.z, i_lo.w, i_hi.x, i_hi.y, i_hi.z, i_hi.w};
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        const char* row = shard + (size_t)ib[m] * ld_bytes;
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+          if (act[r]) cp_async16(stage + (size_t)m * row_bytes + ((size_t)r * 32 + lane) * 16, row + ((size_t)r * 32 + lane) * 16);
+      }
+    }
+    cp_async_commit();
+  };
+
+  uint4 id_lo = make_uint4(0, 0, 0, 0), id_hi = make_uint4(0, 0, 0, 0);
+  for (int s = 0; s < S; ++s) {
+    load_ids(s, id_lo, id_hi);
+    prefetch_block(s, s, id_lo, id_hi);
+  }
+  load_ids(S, id_lo, id_hi);
+  float y_nxt = 0.0f;
+  uint32_t id_nxt = 0u;
+  if (nb > 0) y_nxt = yshard[idx[n]];
+  if (nb > 1) id_nxt = idx[B + n];
+
+  int st = 0;
+  for (long long b = 0; b < nb; ++b) {
+    const int nv = (int)((n_run - b * B) < (long long)B ? (n_run - b * B) : (long long)B);
+    const float y_cur = y_nxt;
+    if (b + 1 < nb) y_nxt = yshard[id_nxt];
+    if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
+    // ---- rows of block b: shared memory -> registers, then refill the stage --------------------------------
+    cp_async_wait(S - 1 < 3 ? S - 1 : 3);  // groups committed: S + b; block b must be complete
+    uint4 raw[R][B];
+    {
+      const unsigned char* stage = ring + (size_t)st * B * row_bytes;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int m = 0; m < B; ++m)
+          raw[r][m] = act[r] ? *(const uint4*)(stage + (size_t)m * row_bytes + ((size_t)r * 32 + lane) * 16)
+                             : make_uint4(0u, 0u, 0u, 0u);
+    }
+    prefetch_block(b + S, st, id_lo, id_hi);
+    load_ids(b + 1 + S, id_lo, id_hi);
+    // ---- G_b and p_b in one pass -----------------------------------------------------------------------
+    float acc[32], accp[B];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+#pragma unroll
+    for (int m = 0; m < B; ++m) accp[m] = 0.0f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+      for (int q = 0; q < QV; ++q) {
+        float x[B][4];
+#pragma unroll
+        for (int m = 0; m < B; ++m) widen_quad<XT>(raw[r][m], q, x[m]);
+#pragma unroll
+        for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+          for (int m = 0; m < n2; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[n2 * (n2 - 1) / 2 + m] = fmaf(x[m][e], x[n2][e], acc[n2 * (n2 - 1) / 2 + m]);
+#pragma unroll
+        for (int m = 0; m < B; ++m)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accp[m] = fmaf(w[r][q * 4 + e], x[m][e], accp[m]);
+      }
+    }
+    const float ptot = warp_transpose_sum8(accp);   // every lane: total of p_{lane >> 2}
+    const float gtot = warp_transpose_sum32(acc);   // lane l: total of Gram entry l
+    // all 28 + 8 totals into every lane (through the warp's scratch line)
+    scratch[lane] = gtot;
+    if ((lane & 3) == 0) scratch[32 + (lane >> 2)] = ptot;
+    __syncwarp();
+    float Gs[BLK_PAIRS], pv[B];
+#pragma unroll
+    for (int i = 0; i < BLK_PAIRS / 4; ++i) {
+      const float4 q = ((const float4*)scratch)[i];
+      Gs[4 * i] = q.x; Gs[4 * i + 1] = q.y; Gs[4 * i + 2] = q.z; Gs[4 * i + 3] = q.w;
+    }
+    {
+      const float4 q0 = ((const float4*)scratch)[8], q1 = ((const float4*)scratch)[9];
+      pv[0] = q0.x; pv[1] = q0.y; pv[2] = q0.z; pv[3] = q0.w; pv[4] = q1.x; pv[5] = q1.y; pv[6] = q1.z; pv[7] = q1.w;
+    }
+    __syncwarp();
+    // ---- 8-step recurrence, every lane the same ----------------------------------------------------------
+    const float a_nv = tab[nv], dl = tab[32 + nv];
+    float t[B], beta[B], yv[B], cf[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m) {
+      yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+      float sc;
+      if (LOSS == LOSS_LOGISTIC) { sc = yv[m] * apw[m] * 1.4426950408889634f; cf[m] = -yv[m] * cfac[m]; }
+      else if (LOSS == LOSS_HINGE) { sc = yv[m] * apw[m]; cf[m] = -yv[m] * cfac[m]; }
+      else { sc = apw[m]; cf[m] = cfac[m]; }
+      if (m >= nv) cf[m] = 0.0f;
+      t[m] = sc * pv[m];
+#pragma unroll
+      for (int k2 = 0; k2 < m; ++k2) Gs[m * (m - 1) / 2 + k2] *= sc;
+    }
+#pragma unroll
+    for (int m = 0; m < B; ++m) {
+      if (LOSS == LOSS_LOGISTIC) {
+        float e, r;
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t[m]));
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+        beta[m] = cf[m] * r;
+      } else if (LOSS == LOSS_HINGE) {
+        beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+      } else {
+        beta[m] = cf[m] * (t[m] - yv[m]);
+      }
+#pragma unroll
+      for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+    }
+    // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m,  gamma_m = beta_m a^nv ----------------------------------
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+      for (int v = 0; v < V; ++v) w[r][v] = fmaf(-dl, w[r][v], w[r][v]);
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        const float gm = beta[m] * a_nv;
+#pragma unroll
+        for (int q = 0; q < QV; ++q) {
+          float x[4];
+          widen_quad<XT>(raw[r][m], q, x);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) w[r][q * 4 + e] = fmaf(-gm, x[e], w[r][q * 4 + e]);
+        }
+      }
+    }
+    st = (st + 1 == S) ? 0 : st + 1;
+  }
+  cp_async_wait(0);
+
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const long long c0 = ((long long)r * 32 + lane) * V;
+    if (act[r]) {
+      float* dst = p.W + (size_t)j * d + c0;
+#pragma unroll
+      for (int v = 0; v < V; ++v) dst[v] = w[r][v];
+    }
+  }
+}
+
+}  // namespace wpsgd

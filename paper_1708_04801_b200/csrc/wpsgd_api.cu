@@ -341,6 +341,51 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
   }
 }
 
+// blocked kernel, one warp per node (small d)
+template <typename XT>
+bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out) {
+  constexpr int V = XVec<XT>::V;
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / V;
+  const int R = (int)((chunks + 31) / 32);
+  if (R > 2) return false;
+  const size_t row_bytes = (size_t)c->d * sizeof(XT);
+  int stages = c->opt_stages > 0 ? c->opt_stages : 3;
+  // two CTAs per SM should fit, so that all of ~7 chains per SM are resident
+  while (stages >= 2 && BlockWarpSmem(stages, row_bytes).total > 100 * 1024) --stages;
+  if (stages < 2) return false;
+  *R_out = R;
+  *stages_out = stages;
+  return true;
+}
+
+template <typename XT, int R>
+wpsgd_status launch_block_warp_r(wpsgd_ctx* c, const BlockParams& bp, size_t smem) {
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<(c->k + BLKW_WARPS - 1) / BLKW_WARPS, 32 * BLKW_WARPS, smem, c->stream>>>(bp);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_block_warp_kernel<XT, R, LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_warp_kernel<XT, R, LOSS_LOGISTIC>);
+    default: return go(chain_block_warp_kernel<XT, R, LOSS_SQUARED>);
+  }
+}
+
+template <typename XT>
+wpsgd_status launch_block_warp(wpsgd_ctx* c, const ChainParams& p, int R, int stages) {
+  BlockParams bp;
+  bp.c = p;
+  bp.stages = stages;
+  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  const size_t smem = BlockWarpSmem(stages, (size_t)c->d * sizeof(XT)).total;
+  return R == 1 ? launch_block_warp_r<XT, 1>(c, bp, smem) : launch_block_warp_r<XT, 2>(c, bp, smem);
+}
+
 template <typename XT>
 wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   constexpr int V = XVec<XT>::V;
@@ -351,11 +396,20 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   int variant = c->opt_variant;
   int bthreads = 0, bR = 0, bstages = 0;
   const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
+  int wR = 0, wstages = 0;
+  const bool block_warp_ok = block_warp_kernel_fits<XT>(c, aligned, &wR, &wstages);
   if (variant == 0) {
     if (!aligned) variant = 1;
-    else if (chunks <= 64) variant = 3;
+    else if (chunks <= 64) variant = block_warp_ok ? 5 : 3;
     else if (block_ok) variant = 4;
     else variant = (chunks > 512 * 4) ? 1 : 2;
+  }
+  if (variant == 5) {
+    if (!block_warp_ok)
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
+                  "eta*lambda <= 0.25");
+    return launch_block_warp<XT>(c, p, wR, wstages);
   }
   if (variant == 4) {
     if (!block_ok)
@@ -543,7 +597,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 4) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..4");
+    if (value < 0 || value > 5) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..5");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");

@@ -154,6 +154,30 @@ def test_blocked_kernel_column_tilings(P, d, bf16, loss):
     assert_parity(P, wl, {"dense_variant": 4})
 
 
+@pytest.mark.parametrize("d,bf16", [(64, False), (200, False), (256, False), (8, False), (72, True), (512, True)])
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("stages", [2, 3])
+def test_blocked_warp_kernel(P, d, bf16, loss, stages):
+    # k = 11: three CTAs of four warps, the last one with an idle warp; step counts with ragged last blocks
+    wl = wi.config5(k=11, d=d, m=40, total_steps=11 * 131, rho=6.0)
+    wl.n_steps[3] = 0
+    wl.n_steps[7] = 5
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    if bf16:
+        wl.X = wl.X.to(torch.bfloat16)
+    wl.w0 = torch.full((d,), 0.05)
+    assert_parity(P, wl, {"dense_variant": 5, "stages": stages})
+
+
+def test_blocked_warp_kernel_limits(P):
+    wl = wi.config2(k=2, d=480, m=16, base_steps=20)  # 120 chunks: too wide for a warp
+    with pytest.raises(P.WpsgdError) as e:
+        gpu_solve(P, wl, {"dense_variant": 5})
+    assert e.value.status_name == "UNSUPPORTED"
+
+
 def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
     wl = wi.config2(k=4, d=1024, m=64, base_steps=100).to("cuda")
     with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
