@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--workload", type=int, default=2, help="benchmark configuration (default 2)")
     ap.add_argument("--rho", type=float, default=4.0, help="speed ratio of workload 5")
     ap.add_argument("--small", action="store_true", help="scaled-down copy of the workload (profiling captures)")
+    ap.add_argument("--rows", type=int, default=0, help="rows per node override (smaller device footprint for profiler captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="name=value passed to wpsgd_set_option")
     return ap.parse_args()
@@ -69,9 +70,11 @@ def make_workload(args, rank: int, device):
     if args.small:
         wl = wi.small(cfg, device=device)
     elif cfg == 5:
-        wl = wi.config5(rho=args.rho, device=device, data_seed=1005 + seed_shift)
+        kw = {"m": args.rows} if args.rows else {}
+        wl = wi.config5(rho=args.rho, device=device, data_seed=1005 + seed_shift, **kw)
     elif cfg in (1, 2, 3, 4):
-        wl = wi.FULL[cfg](device=device, data_seed=1000 + cfg + seed_shift)
+        kw = {"m": args.rows} if args.rows else {}
+        wl = wi.FULL[cfg](device=device, data_seed=1000 + cfg + seed_shift, **kw)
     else:
         raise SystemExit(f"unknown workload {cfg}")
     return wl

@@ -32,8 +32,10 @@ namespace wpsgd {
 
 struct BlockParams {
   ChainParams c;
-  int stages;        // S: blocks in the shared-memory ring (>= 2)
-  double eta_lambda; // eta * lambda in fp64
+  int stages;            // S: blocks in the shared-memory ring (>= 2)
+  double eta_lambda;     // eta * lambda in fp64
+  long long spin_limit;  // polls after which a wait on arriving rows gives up
+  long long drop_block;  // test hook: the rows of this block are never requested (-1: none)
 };
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
@@ -53,6 +55,40 @@ __device__ __forceinline__ void cp_async_wait(int pending) {
     case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
     default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
   }
+}
+
+// ---- bulk asynchronous copies (TMA, untiled form) completing on a shared-memory barrier ------------------------
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(a), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(a), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait for the phase with the given parity to complete; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, uint32_t parity, long long limit) {
+  for (long long i = 0; i < limit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// One contiguous global -> shared copy (no multicast); bytes a multiple of 16, both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_copy_g2s(void* smem_dst, const void* gmem_src, uint32_t bytes, unsigned long long* bar) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst), b = (uint32_t)__cvta_generic_to_shared(bar);
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(d),
+               "l"(gmem_src), "r"(bytes), "r"(b)
+               : "memory");
 }
 
 // Quad q (4 consecutive columns) of a 16-byte chunk, widened to fp32.
@@ -107,40 +143,64 @@ __device__ __forceinline__ float warp_transpose_sum8(float (&v)[8]) {
   return t;
 }
 
+// 8x8 b16 tiles from shared memory, four at a time (lanes 8i..8i+7 give the row addresses of tile i); each
+// lane receives, per tile, the pair of elements (row = lane / 4, columns 2 (lane % 4), +1).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_ptr) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(a)
+               : "memory");
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col). bf16 products are exact in fp32.
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                  uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 constexpr int BLK_B = 8;                           // samples per block
 constexpr int BLK_PAIRS = BLK_B * (BLK_B - 1) / 2;  // 28 Gram entries below the diagonal
-constexpr int BLK_MAX_MATH_WARPS = 8;
+constexpr int BLK_MAX_MATH_WARPS = 16;
 
 // Shared-memory carve-up (bytes). Ring first (16-byte aligned), then the small arrays.
 struct BlockSmem {
-  size_t ring, redG, redP, totG, gam, tab, total;
+  size_t ring, redG, redP, totG, gam, tab, bars, flag, total;
   __host__ __device__ BlockSmem(int stages, size_t row_bytes, int math_warps) {
     ring = 0;
     redG = ring + (size_t)stages * BLK_B * row_bytes;
     (void)math_warps;  // the partial-sum arrays always have room for the maximum number of math warps
-    redP = redG + (size_t)BLK_MAX_MATH_WARPS * 32 * sizeof(float);
+    redP = redG + (size_t)BLK_MAX_MATH_WARPS * 64 * sizeof(float);
     totG = redP + (size_t)BLK_MAX_MATH_WARPS * BLK_B * sizeof(float);
-    gam = totG + 32 * sizeof(float);
+    gam = totG + 64 * sizeof(float);
     tab = gam + 16 * sizeof(float);
-    total = tab + 3 * 16 * sizeof(float);
+    bars = (tab + 3 * 16 * sizeof(float) + 7) / 8 * 8;  // one arrival barrier per ring stage (up to 8)
+    flag = bars + 8 * sizeof(unsigned long long);
+    total = flag + 16;
   }
 };
 
-template <typename XT, int R, int LOSS, bool OVERLAP>
-__global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_kernel(const BlockParams bp) {
+template <typename XT, int R, int LOSS, bool OVERLAP, int MAXW>
+__global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;   // columns per 16-byte chunk
   constexpr int QV = V / 4;        // quads per chunk
   constexpr int B = BLK_B;
   extern __shared__ __align__(16) unsigned char smem[];
   const ChainParams& p = bp.c;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int math_warps = (blockDim.x >> 5) - 1;
+  const int math_warps = (blockDim.x >> 5) - 2;  // warp 0: recurrence, warp 1: row copies, the rest: math
   const int TM = math_warps * 32;
   const int S = bp.stages;
   const int j = p.order[blockIdx.x];
   const long long n_run = p.n_steps[j];
   const long long d = p.d;
-  const size_t row_bytes = (size_t)d * sizeof(XT);  // bytes of a row that are staged
+  // bf16 rows: the Gram block comes from the tensor cores (exact products, fp32 sums), which read 8x8 tiles
+  // across the 8 rows; 16 bytes of padding per staged row keep those reads free of bank conflicts
+  constexpr bool USE_MMA = (sizeof(XT) == 2);
+  constexpr int GW = USE_MMA ? 64 : 32;             // Gram partials per math warp
+  const size_t row_bytes = (size_t)d * sizeof(XT) + (USE_MMA ? 16 : 0);  // stride of a staged row
   const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
   const BlockSmem L(S, row_bytes, math_warps);
   unsigned char* ring = smem + L.ring;
@@ -149,6 +209,8 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
   float* totG = (float*)(smem + L.totG);   // [32] Gram entries summed over the math warps
   float* gam = (float*)(smem + L.gam);     // gamma_0..7, [8] = 1 - a^nv
   float* tab = (float*)(smem + L.tab);     // [0..8] a^k, [16..24] eta / a^{k+1}, [32..40] 1 - a^k
+  unsigned long long* bars = (unsigned long long*)(smem + L.bars);  // bars[s]: rows of the block in stage s have landed
+  volatile int* give_up = (volatile int*)(smem + L.flag);           // set when a bounded wait ran out
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes;
   const float* yshard = p.y + p.shard_off[j];
   const uint32_t* idx = p.idx + p.idx_off[j];  // padded to a multiple of B entries, all valid rows
@@ -162,6 +224,12 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     tab[16 + threadIdx.x] = (float)((double)p.eta0 / (pw * a));
     tab[32 + threadIdx.x] = (float)(1.0 - pw);
   }
+  if (threadIdx.x == 32) {
+    for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
+    *give_up = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();  // tables and barriers are set up
 
   if (warp == 0) {
     // =========================== serial warp ===========================================================
@@ -169,9 +237,9 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     // shuffle inside the dependent chain); lanes only differ in which partial sums they add up and in
     // which gamma they store. Lane n & 7 looks after the label of sample n.
     const int n = lane & (B - 1);
-    for (int i = lane; i < BLK_MAX_MATH_WARPS * 32; i += 32)  // unused partial-sum slots read as zero
-      if (i >= math_warps * 32) redG[i] = 0.0f;
-    for (int i = lane; i < BLK_MAX_MATH_WARPS * B; i += 32)
+    for (int i = lane; i < MAXW * GW; i += 32)  // unused partial-sum slots read as zero
+      if (i >= math_warps * GW) redG[i] = 0.0f;
+    for (int i = lane; i < MAXW * B; i += 32)
       if (i >= math_warps * B) redP[i] = 0.0f;
     // label pipeline in registers: label of block b+1 and sample id of block b+2 are in flight during block b
     float y_nxt = 0.0f;
@@ -209,29 +277,60 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
       }
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       auto gather_gram = [&]() {
-        float gp[BLK_MAX_MATH_WARPS];
+        if (USE_MMA) {
+          // partials are full 8x8 blocks (row-major, symmetric); lane l sums entries l and l + 32
+          float g0[MAXW], g1[MAXW];
 #pragma unroll
-        for (int w = 0; w < BLK_MAX_MATH_WARPS; ++w) gp[w] = redG[w * 32 + lane];
-        totG[lane] = ((gp[0] + gp[1]) + (gp[2] + gp[3])) + ((gp[4] + gp[5]) + (gp[6] + gp[7]));
-        __syncwarp();
+          for (int w = 0; w < MAXW; ++w) { g0[w] = redG[w * 64 + lane]; g1[w] = redG[w * 64 + 32 + lane]; }
 #pragma unroll
-        for (int i = 0; i < BLK_PAIRS / 4; ++i) {
-          const float4 q = ((const float4*)totG)[i];
-          Gs[4 * i] = q.x; Gs[4 * i + 1] = q.y; Gs[4 * i + 2] = q.z; Gs[4 * i + 3] = q.w;
+          for (int h = MAXW / 2; h >= 1; h >>= 1)
+#pragma unroll
+            for (int w = 0; w < h; ++w) { g0[w] += g0[w + h]; g1[w] += g1[w + h]; }
+          totG[lane] = g0[0];
+          totG[32 + lane] = g1[0];
+          __syncwarp();
+#pragma unroll
+          for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+            for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] = totG[n2 * 8 + m] * sc[n2];
+          __syncwarp();
+        } else {
+          float gp[MAXW];
+#pragma unroll
+          for (int w = 0; w < MAXW; ++w) gp[w] = redG[w * 32 + lane];
+#pragma unroll
+          for (int h = MAXW / 2; h >= 1; h >>= 1)
+#pragma unroll
+            for (int w = 0; w < h; ++w) gp[w] += gp[w + h];
+          totG[lane] = gp[0];
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < BLK_PAIRS / 4; ++i) {
+            const float4 q = ((const float4*)totG)[i];
+            Gs[4 * i] = q.x; Gs[4 * i + 1] = q.y; Gs[4 * i + 2] = q.z; Gs[4 * i + 3] = q.w;
+          }
+          __syncwarp();
+#pragma unroll
+          for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+            for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] *= sc[n2];
         }
-        __syncwarp();
-#pragma unroll
-        for (int n2 = 1; n2 < B; ++n2)
-#pragma unroll
-          for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] *= sc[n2];
       };
       if (OVERLAP) gather_gram();  // G_b was finished by the math warps during the previous block
       __syncthreads();             // barrier 1: p_b partials (and, without overlap, G_b partials) are in place
+      // A wait that ran out is flagged before barrier 1 (before barrier 2 in the overlapped schedule); every warp
+      // reads the flag right after that barrier and nothing writes it again before all have read it, so all
+      // warps leave the loop at the same point and no barrier is left waiting.
+      if (!OVERLAP && *give_up) break;
       if (!OVERLAP) gather_gram();
-      float pp[BLK_MAX_MATH_WARPS];
+      float pp[MAXW];
 #pragma unroll
-      for (int w = 0; w < BLK_MAX_MATH_WARPS; ++w) pp[w] = redP[w * B + n];
-      const float psum = ((pp[0] + pp[1]) + (pp[2] + pp[3])) + ((pp[4] + pp[5]) + (pp[6] + pp[7]));
+      for (int w = 0; w < MAXW; ++w) pp[w] = redP[w * B + n];
+#pragma unroll
+      for (int h = MAXW / 2; h >= 1; h >>= 1)
+#pragma unroll
+        for (int w = 0; w < h; ++w) pp[w] += pp[w + h];
+      const float psum = pp[0];
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
@@ -257,12 +356,76 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
         if (lane == m) mine = beta[m] * a_nv;
       if (lane <= B) gam[lane] = mine;
       __syncthreads();  // barrier 2: gamma published
+      if (OVERLAP && *give_up) break;
+    }
+    return;
+  }
+
+  if (warp == 1) {
+    // =========================== copy warp ==============================================================
+    // Lane m < 8 requests row m of a block as one bulk copy; the eight copies complete on the stage's barrier.
+    // A stage is refilled only after a CTA barrier that every reader of its previous content has passed.
+    const uint32_t copy_bytes = (uint32_t)((size_t)d * sizeof(XT));
+    uint32_t id_next = 0u;  // sample id of this lane's row in the next block to request
+    auto peek = [&](long long blk) {
+      if (lane < B && blk < nb) id_next = idx[blk * B + lane];
+    };
+    auto request = [&](long long blk, int stg) {
+      if (blk < nb && blk != bp.drop_block) {
+        if (lane == 0) mbar_arrive_expect_tx(&bars[stg], B * copy_bytes);
+        __syncwarp();
+        if (lane < B)
+          bulk_copy_g2s(ring + ((size_t)stg * B + lane) * row_bytes, shard + (size_t)id_next * ld_bytes, copy_bytes, &bars[stg]);
+      }
+    };
+    long long requested = 0;  // blocks 0 .. requested-1 have been asked for
+    for (int s = 0; s < S; ++s) {
+      peek(s);
+      request(s, s);
+      ++requested;
+    }
+    peek(requested);
+    __syncthreads();  // pairs with the other warps' start-up barrier
+    int st = 0;
+    long long b = 0;
+    if (OVERLAP) {
+      // block 0 went to registers before the start-up barrier: stage 0 takes block S now
+      request(requested, 0);
+      ++requested;
+      peek(requested);
+      st = (S > 1) ? 1 : 0;
+    }
+    bool stop = false;
+    for (; b < nb; ++b) {
+      __syncthreads();  // barrier 1
+      if (!OVERLAP) {
+        if (*give_up) { stop = true; break; }
+        request(requested, st);  // every math warp has block b in registers: its stage takes block b + S
+        ++requested;
+        peek(requested);
+      }
+      __syncthreads();  // barrier 2
+      if (OVERLAP) {
+        if (*give_up) { stop = true; break; }
+        request(requested, st);  // block b+1 went to registers between the barriers: its stage takes block b+1+S
+        ++requested;
+        peek(requested);
+      }
+      st = (st + 1 == S) ? 0 : st + 1;
+    }
+    if (stop) {
+      // leave no copy in flight into this CTA's shared memory: wait (bounded) on the stage of every block that
+      // was requested and may not have landed yet
+      long long blk = b - 1 > 0 ? b - 1 : 0;
+      for (; blk < requested && blk < nb; ++blk)
+        if (blk != bp.drop_block) mbar_wait_bounded(&bars[blk % S], (uint32_t)((blk / S) & 1), bp.spin_limit);
     }
     return;
   }
 
   // ============================= math warps ==============================================================
-  const int tm = threadIdx.x - 32;
+  const int tm = threadIdx.x - 64;
+  const int mw = warp - 2;  // math warp number
   bool act[R];
   float w[R][V];
 #pragma unroll
@@ -280,28 +443,12 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     }
   }
 
-  // sample ids of a block: 8 consecutive entries, 32-byte aligned (every node's stream starts on a multiple of 8)
-  auto load_ids = [&](long long blk, uint4& lo, uint4& hi) {
-    if (blk < nb) {
-      const uint4* q = (const uint4*)(idx + blk * B);
-      lo = __ldg(q);
-      hi = __ldg(q + 1);
+  // wait (bounded) until the rows of block blk have landed in their stage
+  auto wait_rows = [&](int stg, uint32_t parity) {
+    if (!mbar_wait_bounded(&bars[stg], parity, bp.spin_limit)) {
+      set_status(p.status, DEV_TIMEOUT, 1, (long long)blockIdx.x);
+      *give_up = 1;
     }
-  };
-  // issue the copies of this thread's chunks of block blk into ring stage stg (one commit group per call)
-  auto prefetch_block = [&](long long blk, int stg, const uint4& i_lo, const uint4& i_hi) {
-    if (blk < nb) {
-      unsigned char* stage = ring + (size_t)stg * B * row_bytes;
-      const uint32_t ib[B] = {i_lo.x, i_lo.y, i_lo.z, i_lo.w, i_hi.x, i_hi.y, i_hi.z, i_hi.w};
-#pragma unroll
-      for (int m = 0; m < B; ++m) {
-        const char* row = shard + (size_t)ib[m] * ld_bytes;
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-          if (act[r]) cp_async16(stage + (size_t)m * row_bytes + ((size_t)r * TM + tm) * 16, row + ((size_t)r * TM + tm) * 16);
-      }
-    }
-    cp_async_commit();
   };
   // this thread's chunks of the 8 rows of a landed block, shared memory -> registers (the only read of them)
   auto load_raw = [&](int stg, uint4 (&raw)[R][B]) {
@@ -342,11 +489,36 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
   };
   auto publish_g = [&](float (&acc)[32]) {
     const float tot = warp_transpose_sum32(acc);
-    redG[(warp - 1) * 32 + lane] = tot;
+    redG[mw * 32 + lane] = tot;
   };
   auto publish_p = [&](float (&accp)[B]) {
     const float ptot = warp_transpose_sum8(accp);
-    if ((lane & 3) == 0) redP[(warp - 1) * B + (lane >> 2)] = ptot;
+    if ((lane & 3) == 0) redP[mw * B + (lane >> 2)] = ptot;
+  };
+  // Gram block of the rows in ring stage stg over this warp's columns, on the tensor cores: per 16 columns one
+  // m16n8k16 with A = the 8 rows (rows 8..15 of the tile zero) and B = the same rows as the "column" operand
+  auto gram_mma = [&](int stg) {
+    float gc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    const unsigned char* stage = ring + (size_t)stg * B * row_bytes;
+    const int row = lane & 7, mi = lane >> 3;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const long long seg0 = ((long long)r * TM + 32 * mw) * 8;  // first column of the warp's segment
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const long long col = seg0 + ks * 32;
+        if (col >= d) break;
+        const long long c = col + mi * 8;
+        uint32_t q[4];
+        ldmatrix_x4(q, stage + (size_t)row * row_bytes + (size_t)(c < d ? c : col) * 2);
+        if (col + 8 >= d) q[1] = 0u;
+        if (col + 16 >= d) q[2] = 0u;
+        if (col + 24 >= d) q[3] = 0u;
+        mma_bf16_m16n8k16(gc, q[0], 0u, q[1], 0u, q[0], q[1]);
+        mma_bf16_m16n8k16(gc, q[2], 0u, q[3], 0u, q[2], q[3]);
+      }
+    }
+    *(float2*)&redG[mw * 64 + (lane >> 2) * 8 + (lane & 3) * 2] = make_float2(gc[0], gc[1]);
   };
   // w <- w - (1 - a^nv) w - sum_m gamma_m x_m with the rows held in raw
   auto update = [&](const uint4 (&raw)[R][B]) {
@@ -370,27 +542,22 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
     }
   };
 
-  uint4 id_lo = make_uint4(0, 0, 0, 0), id_hi = make_uint4(0, 0, 0, 0);
-  for (int s = 0; s < S; ++s) {
-    load_ids(s, id_lo, id_hi);
-    prefetch_block(s, s, id_lo, id_hi);
-  }
-  load_ids(S, id_lo, id_hi);
   float acc[32], accp[B];
 
   if (OVERLAP) {
     // Two register copies of row blocks: `cur` (block b: p_b, update) and `nxt` (block b+1: G_{b+1}).
     uint4 cur[R][B], nxt[R][B];
-    cp_async_wait(S - 1 < 3 ? S - 1 : 3);  // block 0 has landed
-    load_raw(0, cur);
-    prefetch_block(S, 0, id_lo, id_hi);    // its stage is free again at once
-    load_ids(S + 1, id_lo, id_hi);
 #pragma unroll
     for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-    products(cur, acc, accp, true, false);
+    if (nb > 0) {
+      wait_rows(0, 0u);
+      load_raw(0, cur);
+      products(cur, acc, accp, true, false);
+    }
     publish_g(acc);
-    __syncthreads();  // tables visible; G_0 partials visible to the serial warp
-    int st = (S > 1) ? 1 : 0;  // ring stage of block b+1
+    __syncthreads();  // start-up barrier: G_0 partials visible to the serial warp, stage 0 free
+    int st = (S > 1) ? 1 : 0;  // ring stage of block b+1 ...
+    uint32_t par = (S > 1) ? 0u : 1u;  // ... and the parity of the barrier phase that brings it
     for (long long b = 0; b < nb; ++b) {
 #pragma unroll
       for (int m = 0; m < B; ++m) accp[m] = 0.0f;
@@ -401,48 +568,50 @@ __global__ void __launch_bounds__(32 + 32 * BLK_MAX_MATH_WARPS, 1) chain_block_k
 #pragma unroll
       for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
       if (b + 1 < nb) {
-        // groups committed so far: S + 1 + b (blocks 0 .. S+b); block b+1 must be complete
-        cp_async_wait(S - 1 < 3 ? S - 1 : 3);
+        wait_rows(st, par);
         load_raw(st, nxt);
         products(nxt, acc, accp, true, false);
       }
-      prefetch_block(b + 1 + S, st, id_lo, id_hi);
-      load_ids(b + 2 + S, id_lo, id_hi);
       publish_g(acc);
-      __syncthreads();  // barrier 2: gamma_b is in gam
+      __syncthreads();  // barrier 2: gamma_b is in gam; the stage of block b+1 is free
+      if (*give_up) break;
       update(cur);
 #pragma unroll
       for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int m = 0; m < B; ++m) cur[r][m] = nxt[r][m];
-      st = (st + 1 == S) ? 0 : st + 1;
+      if (++st == S) { st = 0; par ^= 1u; }
     }
   } else {
     // One register copy: the block is read once, G_b and p_b are formed in the same pass over it, and the
     // rows stay in registers across the serial phase for the update.
     uint4 cur[R][B];
-    __syncthreads();  // tables visible
-    int st = 0;       // ring stage of block b
+    __syncthreads();  // start-up barrier
+    int st = 0;       // ring stage of block b ...
+    uint32_t par = 0u;  // ... and the parity of the barrier phase that brings it
     for (long long b = 0; b < nb; ++b) {
-      // groups committed so far: S + b (blocks 0 .. S+b-1); block b must be complete
-      cp_async_wait(S - 1 < 3 ? S - 1 : 3);
+      wait_rows(st, par);
       load_raw(st, cur);
-      prefetch_block(b + S, st, id_lo, id_hi);
-      load_ids(b + 1 + S, id_lo, id_hi);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
 #pragma unroll
       for (int m = 0; m < B; ++m) accp[m] = 0.0f;
-      products(cur, acc, accp, true, true);
-      publish_p(accp);
-      publish_g(acc);
-      __syncthreads();  // barrier 1
+      if (USE_MMA) {
+        gram_mma(st);
+        products(cur, acc, accp, false, true);
+        publish_p(accp);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+        products(cur, acc, accp, true, true);
+        publish_p(accp);
+        publish_g(acc);
+      }
+      __syncthreads();  // barrier 1: the stage of block b is free
+      if (*give_up) break;
       __syncthreads();  // barrier 2: gamma_b is in gam
       update(cur);
-      st = (st + 1 == S) ? 0 : st + 1;
+      if (++st == S) { st = 0; par ^= 1u; }
     }
   }
-  cp_async_wait(0);
 
 #pragma unroll
   for (int r = 0; r < R; ++r) {

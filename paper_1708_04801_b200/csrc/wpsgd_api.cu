@@ -59,7 +59,8 @@ struct wpsgd_ctx {
   // options
   int opt_stages = 0;
   int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_block_rows = 0, opt_cluster = 0, opt_sparse_threads = 32;
-  long long opt_spin_limit = 1ll << 22;
+  long long opt_spin_limit = 1ll << 20;
+  long long opt_drop_block = -1;
   int opt_timing = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   bool ev_valid = false;
@@ -297,20 +298,25 @@ bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* 
   if (!aligned || c->sched != WPSGD_LR_CONST) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;  // keeps a^-8 harmless in fp32
   const long long chunks = c->d / V;
-  const int math_threads = (int)std::min<long long>(32 * BLK_MAX_MATH_WARPS, (chunks + 31) / 32 * 32);
+  // up to 8 math warps with one chunk per thread (two register copies of a block: Gram products overlap the
+  // recurrence); wider rows take up to 16 math warps, then two chunks per thread
+  int max_threads = chunks <= 256 ? 256 : 512;
+  if (c->opt_threads >= 64 && c->opt_threads % 32 == 0) max_threads = std::min(512, c->opt_threads);
+  const int math_threads = (int)std::min<long long>(max_threads, (chunks + 31) / 32 * 32);
   int R = (int)((chunks + math_threads - 1) / math_threads);
   if (R > 2) return false;  // beyond two chunks per thread the rows of a block no longer fit in registers
-  const size_t row_bytes = (size_t)c->d * sizeof(XT);
+  const size_t row_bytes = (size_t)c->d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0);  // bf16 rows are staged with padding
   int stages = c->opt_stages > 0 ? c->opt_stages : 4;
+  if (stages > 8) stages = 8;
   while (stages >= 2 && BlockSmem(stages, row_bytes, math_threads / 32).total > kSmemBudget) --stages;
   if (stages < 2) return false;
-  *threads_out = math_threads + 32;
+  *threads_out = math_threads + 64;
   *R_out = R;
   *stages_out = stages;
   return true;
 }
 
-template <typename XT, int R>
+template <typename XT, int R, bool OVL, int MAXW>
 wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, size_t smem) {
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -322,9 +328,9 @@ wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, si
   switch (c->loss) {
     // one 16-byte chunk per thread: room for two register copies of a block, so the Gram products of the
     // next block overlap the serial recurrence; more chunks: one copy, Gram and p in the same pass
-    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, R == 1>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, R == 1>);
-    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, R == 1>);
+    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, OVL, MAXW>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, OVL, MAXW>);
+    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, OVL, MAXW>);
   }
 }
 
@@ -334,11 +340,15 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
   bp.c = p;
   bp.stages = stages;
   bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
-  const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT), threads / 32 - 1).total;
-  switch (R) {
-    case 1: return launch_block_r<XT, 1>(c, bp, threads, smem);
-    default: return launch_block_r<XT, 2>(c, bp, threads, smem);
-  }
+  bp.spin_limit = c->opt_spin_limit;
+  bp.drop_block = c->opt_drop_block;
+  const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0), threads / 32 - 2).total;
+  const bool wide = threads > 64 + 32 * 8;  // more than 8 math warps: registers allow one copy of a block only
+  constexpr bool kOverlap = sizeof(XT) == 4;  // bf16: the Gram block comes from the tensor cores, nothing to hide
+  if (R == 1) return wide ? launch_block_r<XT, 1, false, 16>(c, bp, threads, smem)
+                          : launch_block_r<XT, 1, kOverlap, 8>(c, bp, threads, smem);
+  return wide ? launch_block_r<XT, 2, false, 16>(c, bp, threads, smem)
+              : launch_block_r<XT, 2, false, 8>(c, bp, threads, smem);
 }
 
 // blocked kernel, one warp per node (small d)
@@ -382,6 +392,8 @@ wpsgd_status launch_block_warp(wpsgd_ctx* c, const ChainParams& p, int R, int st
   bp.c = p;
   bp.stages = stages;
   bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  bp.spin_limit = c->opt_spin_limit;
+  bp.drop_block = -1;
   const size_t smem = BlockWarpSmem(stages, (size_t)c->d * sizeof(XT)).total;
   return R == 1 ? launch_block_warp_r<XT, 1>(c, bp, smem) : launch_block_warp_r<XT, 2>(c, bp, smem);
 }
@@ -620,6 +632,8 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "timing") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "timing must be 0 or 1");
     c->opt_timing = (int)value;
+  } else if (n == "test_drop_block") {
+    c->opt_drop_block = value;
   } else if (n == "spin_limit") {
     if (value < 1) return fail(c, WPSGD_ERR_INVALID_ARG, "spin_limit must be >= 1");
     c->opt_spin_limit = value;

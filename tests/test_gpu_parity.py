@@ -178,6 +178,31 @@ def test_blocked_warp_kernel_limits(P):
     assert e.value.status_name == "UNSUPPORTED"
 
 
+@pytest.mark.parametrize("d,bf16", [(1024, False), (2048, False), (4096, True)])
+def test_bounded_wait_for_rows_reports_timeout_and_context_survives(P, d, bf16):
+    # Failure detection without a fault: the rows of block 3 are never requested (test hook), so the bounded
+    # wait for them runs out; the kernel flags it, leaves in step and returns, and the next run is clean.
+    wl_cpu = wi.config2(k=3, d=d, m=32, base_steps=120)
+    if bf16:
+        wl_cpu.X = wl_cpu.X.to(torch.bfloat16)
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("dense_variant", 4)
+        ctx.set_option("spin_limit", 2000)
+        ctx.set_option("test_drop_block", 3)
+        ctx.run_workload(wl)
+        with pytest.raises(P.WpsgdError) as e:
+            ctx.check()
+        assert e.value.status_name == "TIMEOUT"
+        ctx.set_option("test_drop_block", -1)
+        ctx.set_option("spin_limit", 1 << 20)
+        ctx.run_workload(wl)
+        v = ctx.combine().cpu().numpy()
+        ctx.check()
+    ov, _, _ = oracle.solve(wl_cpu)
+    assert rel_l2(v, ov) <= 1e-4
+
+
 def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
     wl = wi.config2(k=4, d=1024, m=64, base_steps=100).to("cuda")
     with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
