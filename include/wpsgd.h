@@ -73,7 +73,8 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
 /* Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
  * with register-held model, 3 warp per node, 4 blocked kernel: 8 samples per synchronisation, CTA per node; 5 the same with a warp per node), "prefetch" (rows in
  * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "stages" (blocks of 8 rows in the shared-memory ring of the blocked kernel; 0 = as many as fit, up to 4), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
- * (polls after which a device-side wait gives up), "test_drop_block" (test hook of the bounded wait: the rows of
+ * (polls after which a device-side wait gives up), "tc_gram" (1: bf16 rows take the 8x8 Gram block of the blocked kernel from mma.sync tensor-core
+ * instructions instead of FFMA; same result up to summation order), "test_drop_block" (test hook of the bounded wait: the rows of
  * that block of every chain are never requested, so the wait for them runs out; -1 = off), "timing" (1: record events around the chain kernel). Unknown name or bad value:
  * WPSGD_ERR_INVALID_ARG. The result of a run never depends on these beyond rounding order. */
 wpsgd_status wpsgd_set_option(wpsgd_ctx* ctx, const char* name, int64_t value);

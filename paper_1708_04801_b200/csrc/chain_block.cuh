@@ -36,6 +36,7 @@ struct BlockParams {
   double eta_lambda;     // eta * lambda in fp64
   long long spin_limit;  // polls after which a wait on arriving rows gives up
   long long drop_block;  // test hook: the rows of this block are never requested (-1: none)
+  const int* group_order;  // warp-per-node kernel: node of every (CTA, warp) slot, -1 = none
 };
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
@@ -182,7 +183,7 @@ struct BlockSmem {
   }
 };
 
-template <typename XT, int R, int LOSS, bool OVERLAP, int MAXW>
+template <typename XT, int R, int LOSS, bool OVERLAP, int MAXW, bool TC_GRAM>
 __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;   // columns per 16-byte chunk
   constexpr int QV = V / 4;        // quads per chunk
@@ -198,9 +199,9 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
   const long long d = p.d;
   // bf16 rows: the Gram block comes from the tensor cores (exact products, fp32 sums), which read 8x8 tiles
   // across the 8 rows; 16 bytes of padding per staged row keep those reads free of bank conflicts
-  constexpr bool USE_MMA = (sizeof(XT) == 2);
+  constexpr bool USE_MMA = TC_GRAM && (sizeof(XT) == 2);
   constexpr int GW = USE_MMA ? 64 : 32;             // Gram partials per math warp
-  const size_t row_bytes = (size_t)d * sizeof(XT) + (USE_MMA ? 16 : 0);  // stride of a staged row
+  const size_t row_bytes = (size_t)d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0);  // stride of a staged row
   const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
   const BlockSmem L(S, row_bytes, math_warps);
   unsigned char* ring = smem + L.ring;
@@ -634,20 +635,20 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
 // ======================================================================================================
 namespace wpsgd {
 
-constexpr int BLKW_WARPS = 4;  // nodes per CTA
+constexpr int BLKW_MAX_WARPS = 4;  // most nodes per CTA
 
 struct BlockWarpSmem {
   size_t ring, scratch, tab, total;
-  __host__ __device__ BlockWarpSmem(int stages, size_t row_bytes) {
+  __host__ __device__ BlockWarpSmem(int stages, size_t row_bytes, int warps) {
     ring = 0;
-    scratch = ring + (size_t)BLKW_WARPS * stages * BLK_B * row_bytes;
-    tab = scratch + (size_t)BLKW_WARPS * 48 * sizeof(float);
+    scratch = ring + (size_t)warps * stages * BLK_B * row_bytes;
+    tab = scratch + (size_t)warps * 48 * sizeof(float);
     total = tab + 3 * 16 * sizeof(float);
   }
 };
 
 template <typename XT, int R, int LOSS>
-__global__ void __launch_bounds__(32 * BLKW_WARPS) chain_block_warp_kernel(const BlockParams bp) {
+__global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;
   constexpr int QV = V / 4;
   constexpr int B = BLK_B;
@@ -658,7 +659,8 @@ __global__ void __launch_bounds__(32 * BLKW_WARPS) chain_block_warp_kernel(const
   const long long d = p.d;
   const size_t row_bytes = (size_t)d * sizeof(XT);
   const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
-  const BlockWarpSmem L(S, row_bytes);
+  const int nwarps = blockDim.x >> 5;
+  const BlockWarpSmem L(S, row_bytes, nwarps);
   unsigned char* ring = smem + L.ring + (size_t)warp * S * B * row_bytes;
   float* scratch = (float*)(smem + L.scratch) + warp * 48;  // [0..27] G entries, [32..39] p
   float* tab = (float*)(smem + L.tab);
@@ -672,9 +674,10 @@ __global__ void __launch_bounds__(32 * BLKW_WARPS) chain_block_warp_kernel(const
     tab[32 + threadIdx.x] = (float)(1.0 - pw);
   }
   __syncthreads();  // the only CTA-wide barrier; every warp passes it exactly once
-  const int slot = (int)blockIdx.x * BLKW_WARPS + warp;
-  if (slot >= p.k) return;
-  const int j = p.order[slot];
+  // slot -> node table (group_order): the nodes of a CTA are chosen on the host so that every CTA carries about
+  // the same total number of steps; -1 marks an unused slot
+  const int j = bp.group_order[(int)blockIdx.x * nwarps + warp];
+  if (j < 0) return;
   const long long n_run = p.n_steps[j];
   const long long nb = (n_run + B - 1) / B;
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes;

@@ -36,6 +36,7 @@ struct wpsgd_ctx {
   long long* t_count = nullptr;      // [k] entries of the sample stream per node (steps rounded up to 8)
   int* t_order = nullptr;            // [k]
   int* t_ids = nullptr;              // [k] node numbers entering the sample stream
+  int* t_group = nullptr;            // [k + 8] node of every (CTA, warp) slot of the warp-per-node blocked kernel
   double* t_weights = nullptr;       // [k]
   uint32_t* idx = nullptr;
   size_t idx_cap = 0;  // entries
@@ -53,6 +54,7 @@ struct wpsgd_ctx {
   bool have_run = false;
   std::vector<long long> steps_done;
   std::vector<int> node_ids;
+  std::vector<long long> last_steps;  // step counts of the launch being prepared
   float eta0 = 0.f, lambda = 0.f;
   int sched = 0, loss = 0;
   uint64_t seed = 0;
@@ -61,6 +63,7 @@ struct wpsgd_ctx {
   int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_block_rows = 0, opt_cluster = 0, opt_sparse_threads = 32;
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
+  int opt_tc_gram = 0;
   int opt_timing = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   bool ev_valid = false;
@@ -316,7 +319,7 @@ bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* 
   return true;
 }
 
-template <typename XT, int R, bool OVL, int MAXW>
+template <typename XT, int R, bool OVL, int MAXW, bool TC>
 wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, size_t smem) {
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -328,9 +331,9 @@ wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, si
   switch (c->loss) {
     // one 16-byte chunk per thread: room for two register copies of a block, so the Gram products of the
     // next block overlap the serial recurrence; more chunks: one copy, Gram and p in the same pass
-    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, OVL, MAXW>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, OVL, MAXW>);
-    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, OVL, MAXW>);
+    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, OVL, MAXW, TC>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, OVL, MAXW, TC>);
+    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, OVL, MAXW, TC>);
   }
 }
 
@@ -342,18 +345,31 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
   bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
   bp.spin_limit = c->opt_spin_limit;
   bp.drop_block = c->opt_drop_block;
+  bp.group_order = nullptr;
   const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0), threads / 32 - 2).total;
   const bool wide = threads > 64 + 32 * 8;  // more than 8 math warps: registers allow one copy of a block only
-  constexpr bool kOverlap = sizeof(XT) == 4;  // bf16: the Gram block comes from the tensor cores, nothing to hide
-  if (R == 1) return wide ? launch_block_r<XT, 1, false, 16>(c, bp, threads, smem)
-                          : launch_block_r<XT, 1, kOverlap, 8>(c, bp, threads, smem);
-  return wide ? launch_block_r<XT, 2, false, 16>(c, bp, threads, smem)
-              : launch_block_r<XT, 2, false, 8>(c, bp, threads, smem);
+  if (sizeof(XT) == 2) {
+    // bf16 rows: one register copy; the Gram block from FFMA (default) or from the tensor cores (option)
+    if (c->opt_tc_gram) {
+      if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, true>(c, bp, threads, smem)
+                              : launch_block_r<XT, 1, false, 8, true>(c, bp, threads, smem);
+      return wide ? launch_block_r<XT, 2, false, 16, true>(c, bp, threads, smem)
+                  : launch_block_r<XT, 2, false, 8, true>(c, bp, threads, smem);
+    }
+    if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, false>(c, bp, threads, smem)
+                            : launch_block_r<XT, 1, false, 8, false>(c, bp, threads, smem);
+    return wide ? launch_block_r<XT, 2, false, 16, false>(c, bp, threads, smem)
+                : launch_block_r<XT, 2, false, 8, false>(c, bp, threads, smem);
+  }
+  if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, false>(c, bp, threads, smem)
+                          : launch_block_r<XT, 1, true, 8, false>(c, bp, threads, smem);
+  return wide ? launch_block_r<XT, 2, false, 16, false>(c, bp, threads, smem)
+              : launch_block_r<XT, 2, false, 8, false>(c, bp, threads, smem);
 }
 
 // blocked kernel, one warp per node (small d)
 template <typename XT>
-bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out) {
+bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
   constexpr int V = XVec<XT>::V;
   if (!aligned || c->sched != WPSGD_LR_CONST) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
@@ -361,20 +377,41 @@ bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* s
   const int R = (int)((chunks + 31) / 32);
   if (R > 2) return false;
   const size_t row_bytes = (size_t)c->d * sizeof(XT);
-  int stages = c->opt_stages > 0 ? c->opt_stages : 3;
-  // two CTAs per SM should fit, so that all of ~7 chains per SM are resident
-  while (stages >= 2 && BlockWarpSmem(stages, row_bytes).total > 100 * 1024) --stages;
-  if (stages < 2) return false;
+  // Four nodes per CTA and two CTAs per SM. Each chain is bound by its own dependent instruction stream, so what
+  // a long chain needs is few co-runners late in the run, not an equal share of work per SM: with chains dealt out
+  // longest first, the CTAs of the longest chains land on the SMs first and are paired with the shortest ones.
+  // (Measured on k = 1024, d = 256, speed ratio 4: 4.9 ms this way, 6.9 ms with one balanced 7-warp CTA per SM.)
+  int warps = (int)std::min<long long>(4, std::max<long long>(1, c->k));
+  if (c->opt_threads >= 32 && c->opt_threads % 32 == 0) warps = std::min(BLKW_MAX_WARPS, c->opt_threads / 32);
+  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 4) : 3;
+  while (BlockWarpSmem(stages, row_bytes, warps).total > (warps <= 4 ? 100 * 1024 : kSmemBudget)) {
+    if (stages > 2) --stages;
+    else if (warps > 1) --warps;
+    else return false;
+  }
   *R_out = R;
   *stages_out = stages;
+  *warps_out = warps;
   return true;
 }
 
+// Nodes of every CTA of the warp-per-node kernel: longest first, consecutive ranks share a CTA; -1 fills the last one.
+wpsgd_status upload_groups(wpsgd_ctx* c, const long long* n_steps_host, int warps, int* ctas_out) {
+  const int k = c->k;
+  const int ctas = (k + warps - 1) / warps;
+  std::vector<int> group((size_t)ctas * warps, -1);
+  std::iota(group.begin(), group.begin() + k, 0);
+  std::stable_sort(group.begin(), group.begin() + k, [&](int a, int b) { return n_steps_host[a] > n_steps_host[b]; });
+  CU_TRY(c, cudaMemcpyAsync(c->t_group, group.data(), group.size() * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  *ctas_out = ctas;
+  return WPSGD_OK;
+}
+
 template <typename XT, int R>
-wpsgd_status launch_block_warp_r(wpsgd_ctx* c, const BlockParams& bp, size_t smem) {
+wpsgd_status launch_block_warp_r(wpsgd_ctx* c, const BlockParams& bp, size_t smem, int ctas, int warps) {
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<(c->k + BLKW_WARPS - 1) / BLKW_WARPS, 32 * BLKW_WARPS, smem, c->stream>>>(bp);
+    kern<<<ctas, 32 * warps, smem, c->stream>>>(bp);
     CU_TRY(c, cudaGetLastError());
     c->launches++;
     return WPSGD_OK;
@@ -387,15 +424,19 @@ wpsgd_status launch_block_warp_r(wpsgd_ctx* c, const BlockParams& bp, size_t sme
 }
 
 template <typename XT>
-wpsgd_status launch_block_warp(wpsgd_ctx* c, const ChainParams& p, int R, int stages) {
+wpsgd_status launch_block_warp(wpsgd_ctx* c, const ChainParams& p, int R, int stages, int warps) {
   BlockParams bp;
   bp.c = p;
   bp.stages = stages;
   bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
   bp.spin_limit = c->opt_spin_limit;
   bp.drop_block = -1;
-  const size_t smem = BlockWarpSmem(stages, (size_t)c->d * sizeof(XT)).total;
-  return R == 1 ? launch_block_warp_r<XT, 1>(c, bp, smem) : launch_block_warp_r<XT, 2>(c, bp, smem);
+  bp.group_order = c->t_group;
+  int ctas = 0;
+  wpsgd_status s = upload_groups(c, c->last_steps.data(), warps, &ctas);
+  if (s != WPSGD_OK) return s;
+  const size_t smem = BlockWarpSmem(stages, (size_t)c->d * sizeof(XT), warps).total;
+  return R == 1 ? launch_block_warp_r<XT, 1>(c, bp, smem, ctas, warps) : launch_block_warp_r<XT, 2>(c, bp, smem, ctas, warps);
 }
 
 template <typename XT>
@@ -408,8 +449,8 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   int variant = c->opt_variant;
   int bthreads = 0, bR = 0, bstages = 0;
   const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
-  int wR = 0, wstages = 0;
-  const bool block_warp_ok = block_warp_kernel_fits<XT>(c, aligned, &wR, &wstages);
+  int wR = 0, wstages = 0, wwarps = 0;
+  const bool block_warp_ok = block_warp_kernel_fits<XT>(c, aligned, &wR, &wstages, &wwarps);
   if (variant == 0) {
     if (!aligned) variant = 1;
     else if (chunks <= 64) variant = block_warp_ok ? 5 : 3;
@@ -421,7 +462,7 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
       return fail(c, WPSGD_ERR_UNSUPPORTED,
                   "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
                   "eta*lambda <= 0.25");
-    return launch_block_warp<XT>(c, p, wR, wstages);
+    return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
   }
   if (variant == 4) {
     if (!block_ok)
@@ -470,6 +511,7 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
   if (pl.total > 0 && (!X || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "X or y is NULL");
   s = upload_plan_and_stream(c, pl);
   if (s != WPSGD_OK) return s;
+  c->last_steps = pl.steps;
   ChainParams p;
   p.X = X; p.ld = ld; p.y = y;
   p.shard_off = c->t_shard_off; p.n_steps = c->t_steps; p.first = c->t_first; p.idx_off = c->t_idx_off;
@@ -506,14 +548,15 @@ struct StaticLayout {
   size_t count = align256(rows + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t order = align256(count + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t ids = align256(order + sizeof(int) * WPSGD_STATIC_MAX_NODES);
-  size_t weights = align256(ids + sizeof(int) * WPSGD_STATIC_MAX_NODES);
+  size_t group = align256(ids + sizeof(int) * WPSGD_STATIC_MAX_NODES);
+  size_t weights = align256(group + sizeof(int) * (WPSGD_STATIC_MAX_NODES + 8));
   size_t scale = align256(weights + sizeof(double) * WPSGD_STATIC_MAX_NODES);
   size_t status = align256(scale + sizeof(double) * WPSGD_STATIC_MAX_NODES);
   size_t total = align256(status + sizeof(DevStatus));
 };
 constexpr size_t kStaticBytes = align256(sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS) +
                                 align256(sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES)) +
-                                12 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
+                                13 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
 constexpr int kStaticMaxDevices = 64;
 }  // namespace
 
@@ -582,6 +625,7 @@ wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, w
   ALLOC(c->t_count, (size_t)k * sizeof(long long));
   ALLOC(c->t_order, (size_t)k * sizeof(int));
   ALLOC(c->t_ids, (size_t)k * sizeof(int));
+  ALLOC(c->t_group, ((size_t)k + 8) * sizeof(int));
   ALLOC(c->t_weights, (size_t)k * sizeof(double));
   ALLOC(c->status, sizeof(DevStatus));
 #undef ALLOC
@@ -595,7 +639,7 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* c) {
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
   void* ptrs[] = {c->W, c->scale, c->t_shard_off, c->t_steps, c->t_first, c->t_idx_off, c->t_rows, c->t_count, c->t_order,
-                  c->t_ids, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0};
+                  c->t_ids, c->t_group, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev0) cudaEventDestroy(c->ev0);
@@ -632,6 +676,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "timing") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "timing must be 0 or 1");
     c->opt_timing = (int)value;
+  } else if (n == "tc_gram") {
+    if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "tc_gram must be 0 or 1");
+    c->opt_tc_gram = (int)value;
   } else if (n == "test_drop_block") {
     c->opt_drop_block = value;
   } else if (n == "spin_limit") {
@@ -923,6 +970,7 @@ wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wp
   c.t_count = (long long*)(base + L.count);
   c.t_order = (int*)(base + L.order);
   c.t_ids = (int*)(base + L.ids);
+  c.t_group = (int*)(base + L.group);
   c.t_weights = (double*)(base + L.weights);
   c.scale = (double*)(base + L.scale);
   c.status = (DevStatus*)(base + L.status);
