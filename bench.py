@@ -36,7 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the chain kernel from an ncu capture, with the hash of the
 # kernel sources the capture was taken from; reported as null once the sources have changed.
-NCU_TRAFFIC = {"config2": {"src_sha": "", "bytes_per_launch": None}}
+NCU_TRAFFIC = {"config2": {"src_sha": "a7e854bd028dfcab", "bytes_per_launch": 601919744}}
 
 
 def parse_args():
@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--rho", type=float, default=4.0, help="speed ratio of workload 5")
     ap.add_argument("--small", action="store_true", help="scaled-down copy of the workload (profiling captures)")
     ap.add_argument("--rows", type=int, default=0, help="rows per node override (smaller device footprint for profiler captures)")
+    ap.add_argument("--also", default="3,5", help="further workloads measured after the main one at 1 GPU and reported "
+                    "under other_workloads (device-resident timing only); empty to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="name=value passed to wpsgd_set_option")
     return ap.parse_args()
@@ -147,6 +149,46 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measure_other(P, args, cfg: int, dev, peak: float):
+    """Device-resident timing of one more workload: chains + combination, 3 warm-up and 3 timed steps."""
+    import argparse as _ap
+
+    import torch
+
+    a2 = _ap.Namespace(**vars(args))
+    a2.workload, a2.small, a2.rows = cfg, False, 0
+    wl = make_workload(a2, 0, dev)
+    with P.Context(wl.k, wl.d, device=dev.index) as ctx:
+        ctx.set_option("timing", 1)
+        v = torch.empty(wl.d, dtype=torch.float32, device=dev)
+        for _ in range(3):
+            ctx.run_workload(wl)
+            ctx.combine(out=v)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        chain = []
+        e0.record()
+        for _ in range(3):
+            ctx.run_workload(wl)
+            ctx.combine(out=v)
+        e1.record()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            ctx.run_workload(wl)
+            chain.append(ctx.last_chain_ms())
+        ctx.check()
+    ms = e0.elapsed_time(e1) / 3
+    cms = float(np.mean(chain))
+    achieved = bytes_per_update(wl) * wl.total_steps / (cms * 1e-3) / 1e9
+    out = {"workload": describe(wl, a2), "value": wl.total_steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+           "steps": 3, "warmup": 3, "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                                                 "frac": achieved / peak, "kernel_ms": cms,
+                                                 "bytes_per_sample_update": bytes_per_update(wl)}}
+    del wl
+    torch.cuda.empty_cache()
+    return out
 
 
 def cpu_baseline(wl_cpu, min_seconds=10.0, max_passes=30):
@@ -298,7 +340,6 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    clocks = sampler.stop() if rank == 0 else None
     ctx.check()
     if world > 1:
         t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
@@ -333,6 +374,7 @@ def main():
                "h2d_bytes_per_step": int(Xh.numel() * Xh.element_size() + yh.numel() * 4) * world,
                "d2h_bytes_per_step": int(wl.d * 4) * world, "steps": n_e2e}
 
+    clocks = sampler.stop() if rank == 0 else None  # sampled across the device-timed and the end-to-end loops
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(peaks_path):
@@ -362,6 +404,20 @@ def main():
                 line["cpu_baseline"] = cpu_baseline(wl_cpu)
             else:
                 line["cpu_baseline"] = None
+        if world == 1 and args.also and not args.small and not args.rows:
+            ctx.destroy()
+            del wl, v
+            torch.cuda.empty_cache()
+            others = []
+            for tok in args.also.split(","):
+                cfg = int(tok)
+                if cfg == args.workload:
+                    continue
+                try:
+                    others.append(measure_other(P, args, cfg, dev, peak))
+                except Exception as exc:  # e.g. not enough device memory for the 32 GiB workload
+                    others.append({"workload": f"config{cfg}", "error": str(exc)[:200]})
+            line["other_workloads"] = others
         print(json.dumps(line), flush=True)
     ctx.destroy()
     if world > 1:
