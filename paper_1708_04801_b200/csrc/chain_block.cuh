@@ -10,19 +10,23 @@
 // not depend on the model at all, so it is computed one block ahead. What stays serial is a scalar
 // recurrence of B steps per block, done by one warp.
 //
-// One CTA per node: warp 0 is the "serial warp" (sums the partial products, runs the B-step
-// recurrence, publishes gamma); the other warps are "math warps", each thread owning fixed columns of
-// the model (in registers) for the whole chain. Rows reach shared memory through a ring of S blocks
-// filled by per-thread 16-byte asynchronous copies: every thread copies exactly the bytes it later
-// reads itself, so the ring needs no barrier and no wait that could hang.
+// One CTA per node: warp 0 is the "recurrence warp" (sums the partial products, runs the B-step recurrence,
+// publishes gamma); warp 1 is the "copy warp" (requests the 8 rows of a future block as bulk asynchronous
+// copies, cp.async.bulk, that complete on a shared-memory barrier of the ring stage; never multicast); the other
+// warps are "math warps", each thread owning fixed columns of the model in registers for the whole chain.
+// A landed block is read from shared memory exactly once, into registers. Every wait on a stage barrier is
+// bounded: when it runs out the kernel records a timeout in the status word, all warps leave the loop at the
+// same barrier, the copy warp waits (bounded again) for copies still in flight, and the kernel returns.
 //
-// Per block b:   math warps                               serial warp
+// Per block b (overlapped schedule, one 16-byte chunk per thread):
+//                math warps                               recurrence warp
 //                p_b partials (needs w)  -> smem          sum G_b partials (written last round)
 //                ------------------------- barrier 1 --------------------------------------
 //                G_{b+1} partials -> smem                 sum p_b, B-step recurrence, gamma -> smem
 //                ------------------------- barrier 2 --------------------------------------
-//                w <- w - (1-a^B) w - sum gamma_m x_m     prefetch labels
-//                prefetch rows of block b+S
+//                w <- w - (1-a^B) w - sum gamma_m x_m     labels and constants of block b+1
+// With two chunks per thread (wide rows) registers hold one block only: G_b and p_b are formed in one pass
+// before barrier 1 and the math warps idle during the recurrence.
 #pragma once
 
 #include "chain_dense.cuh"
