@@ -57,8 +57,22 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
   const float* yshard = p.y + p.shard_off[j];
   const uint32_t* idx = p.idx + p.idx_off[j];
   float* u = p.U + (size_t)j * p.d;
-  double sc = 1.0;
+  // The scale factor does not depend on the data: s_n = prod_{q<=n} (1 - eta_q lambda). It is advanced in fp64
+  // ahead of the chain, together with the rows, and handed to the step as two floats (s before the step, and
+  // eta_n / s after it), so that no fp64 division or square root sits on the serial path.
+  double sc = 1.0;  // scale after the last step whose constants have been prepared
   const double lam = (double)p.lambda, eta0 = (double)p.eta0;
+  auto prepare_scalars = [&](long long step0, float& s_before, float& eta_over_s, float& fold) {
+    fold = 0.0f;
+    if (sc < 1e-12) {  // fold the scale into u at this step, before fp32 range is at risk
+      fold = (float)sc;
+      sc = 1.0;
+    }
+    s_before = (float)sc;
+    const double eta = p.sched == LR_INV_SQRT ? eta0 / sqrt((double)(step0 + 1)) : eta0;
+    sc *= (1.0 - eta * lam);
+    eta_over_s = (float)(eta / sc);
+  };
 
   // rings (slot = step mod P): sample id of step s+3P; extents+label of step s+2P... see refill below
   uint32_t ib[P];
@@ -69,17 +83,20 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
   float yb[P];
   int cb[P][Q];
   float vb[P][Q];
+  float scb[P], cfb[P], fob[P];
 
   // prologue: bring the three pipeline levels up (dependent loads, paid once)
 #pragma unroll
   for (int t = 0; t < P; ++t) {
     ib[t] = 0u; ra0[t] = 0; ra1[t] = 0; ya[t] = 0.0f; sb[t] = 0; nb[t] = 0; yb[t] = 0.0f;
+    scb[t] = 1.0f; cfb[t] = 0.0f; fob[t] = 0.0f;
 #pragma unroll
     for (int q = 0; q < Q; ++q) { cb[t][q] = 0; vb[t][q] = 0.0f; }
     if (t < n_run) {
       const uint32_t i0 = idx[t];
       const long long b = rp[i0], e = rp[i0 + 1];
       sb[t] = b; nb[t] = (int)(e - b); yb[t] = yshard[i0];
+      prepare_scalars(t, scb[t], cfb[t], fob[t]);
 #pragma unroll
       for (int q = 0; q < Q; ++q) {
         const int o = lane + 32 * q;
@@ -106,11 +123,21 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
       float v[Q];
 #pragma unroll
       for (int q = 0; q < Q; ++q) { c[q] = cb[t][q]; v[q] = vb[t][q]; }
-      // ---- refill the three levels of slot t ------------------------------------------------------
+      const float s_before = scb[t], eta_over_s = cfb[t], fold = fob[t];
+      if (fold != 0.0f) {  // rare: the scale was folded back at this step
+        for (long long cc = lane; cc < p.d; cc += 32) u[cc] *= fold;
+        __syncwarp();
+      }
+      // ---- margin -------------------------------------------------------------------------------
+      float uq[Q];
+#pragma unroll
+      for (int q = 0; q < Q; ++q) uq[q] = (lane + 32 * q < nnz) ? u[c[q]] : 0.0f;  // gathers in flight ...
+      // ---- ... while the three levels of slot t are refilled ------------------------------------------------------
       if (s + P < n_run) {
         const long long b = ra0[t];
         const int cnt = (int)(ra1[t] - b);
         sb[t] = b; nb[t] = cnt; yb[t] = ya[t];
+        prepare_scalars(s + P, scb[t], cfb[t], fob[t]);
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
           const int o = lane + 32 * q;
@@ -123,26 +150,16 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
       }
       if (s + 3 * P < n_run) ib[t] = idx[s + 3 * P];
 
-      // ---- margin -------------------------------------------------------------------------------
-      float uq[Q];
       float acc = 0.0f;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) {
-        uq[q] = 0.0f;
-        if (lane + 32 * q < nnz) {
-          uq[q] = u[c[q]];
-          acc = fmaf(uq[q], v[q], acc);
-        }
-      }
+      for (int q = 0; q < Q; ++q) acc = fmaf(uq[q], v[q], acc);
       for (int o = lane + 32 * Q; o < nnz; o += 32) acc = fmaf(u[p.col_idx[beg + o]], p.val[beg + o], acc);
       acc = warp_sum(acc);
-      const float z = (float)(sc * (double)acc);
+      const float z = s_before * acc;
       const float g = loss_derivative(p.loss, yv, z);
-      const double eta = p.sched == LR_INV_SQRT ? eta0 / sqrt((double)(s + 1)) : eta0;
-      sc *= (1.0 - eta * lam);
-      // ---- loss term on the row's nonzeros ---------------------------------------------------------
+      // ---- loss term on the row's nonzeros: u_c <- u_c - (eta_n g / s_n) x_c -----------------------------
       if (g != 0.0f) {
-        const float coef = (float)(eta * (double)g / sc);
+        const float coef = eta_over_s * g;
 #pragma unroll
         for (int q = 0; q < Q; ++q)
           if (lane + 32 * q < nnz) u[c[q]] = fmaf(-coef, v[q], uq[q]);
@@ -150,12 +167,6 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
           const int cc = p.col_idx[beg + o];
           u[cc] = fmaf(-coef, p.val[beg + o], u[cc]);
         }
-      }
-      if (sc < 1e-12) {  // fold the scale into u before fp32 range is at risk
-        __syncwarp();
-        const float f = (float)sc;
-        for (long long cc = lane; cc < p.d; cc += 32) u[cc] *= f;
-        sc = 1.0;
       }
       __syncwarp();  // the next step's gathers must see this step's scatters
     }
