@@ -70,7 +70,13 @@ wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, w
 /* Release everything the context owns. Synchronises the stream first. NULL is accepted. */
 wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
 
-/* Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
+/* Options by name. "sampling": order of the examples. 0 (default) = independent uniform draws as described in the
+ * header comment. 1 = the literal reading of Algorithm 1 ("randomly shuffle the data on machine i", then "get the
+ * n-th example"): one fixed pseudo-random permutation pi_j of the shard per node, cycled, i.e. the n-th example
+ * is row pi_j((n-1) mod m_j); pi_j is a 4-round balanced Feistel network on the even bit count covering m_j - 1
+ * with cycle walking, keyed by the Philox block at counter (0, 0, j, 1) under the seed, round function
+ * mix(R ^ key) = multiply 0x85EBCA6B, xor-shift 13, multiply 0xC2B2AE35, xor-shift 16, masked to half the bits.
+ * Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
  * with register-held model, 3 warp per node, 4 blocked kernel: 8 samples per synchronisation, CTA per node; 5 the same with a warp per node), "prefetch" (rows in
  * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "stages" (blocks of 8 rows in the shared-memory ring of the blocked kernel; 0 = as many as fit, up to 4), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
  * (polls after which a device-side wait gives up), "tc_gram" (1: bf16 rows take the 8x8 Gram block of the blocked kernel from mma.sync tensor-core

@@ -78,6 +78,12 @@ def _np(a, dtype):
     return a
 
 
+def set_sampling(mode: int):
+    """0: i.i.d. uniform draws (default); 1: one fixed shuffle per node, cycled. Applies to later calls."""
+    if lib().oracle_set_sampling(int(mode)):
+        raise ValueError("unknown sampling mode")
+
+
 def philox4x32_10(ctr, key):
     c = np.asarray(ctr, dtype=np.uint32)
     k = np.asarray(key, dtype=np.uint32)

@@ -81,6 +81,52 @@ inline uint32_t sample_index(uint64_t seed, uint32_t node, int64_t n /*1-based*/
     return (uint32_t)(((uint64_t)u * m) >> 32);
 }
 
+// Alternative sample order, the literal reading of Algorithm 1 ("randomly shuffle the data on machine i", then
+// "get the n-th example"): one fixed pseudo-random permutation pi_j of the shard's m rows per node, cycled when
+// a node runs more than m steps: the n-th example is row pi_j((n-1) mod m).
+// pi_j is a keyed bijection of [0, m): a 4-round balanced Feistel network on 2w bits (2w = the even number of
+// bits >= 2 that covers m-1) with cycle walking (re-encrypt until the value is < m). Round keys: the four
+// output words of Philox4x32-10 at counter (0, 0, j, 1) under the seed. Round function: xor with the key,
+// multiply by 0x85EBCA6B, xor-shift 13, multiply by 0xC2B2AE35, xor-shift 16 (a 32-bit integer mixer), masked
+// to w bits.
+inline uint32_t mix32(uint32_t x, uint32_t key) {
+    uint32_t h = x ^ key;
+    h *= 0x85EBCA6Bu;
+    h ^= h >> 13;
+    h *= 0xC2B2AE35u;
+    h ^= h >> 16;
+    return h;
+}
+
+inline uint32_t shuffled_index(uint64_t seed, uint32_t node, int64_t n /*1-based*/, uint64_t m) {
+    if (m <= 1) return 0;
+    U4 c;
+    c.v[0] = 0; c.v[1] = 0; c.v[2] = node; c.v[3] = 1;
+    const U4 keys = philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    int bits = 0;
+    while (((uint64_t)1 << bits) < m) ++bits;   // smallest bits with 2^bits >= m
+    if (bits < 2) bits = 2;
+    if (bits & 1) ++bits;
+    const int w = bits / 2;
+    const uint32_t mask = (w == 16) ? 0xFFFFu : (((uint32_t)1 << w) - 1u);
+    uint64_t x = (uint64_t)((n - 1) % (int64_t)m);
+    do {
+        uint32_t L = (uint32_t)(x >> w), R = (uint32_t)x & mask;
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t t = (L ^ mix32(R, keys.v[i])) & mask;
+            L = R;
+            R = t;
+        }
+        x = ((uint64_t)L << w) | R;
+    } while (x >= m);
+    return (uint32_t)x;
+}
+
+// sampling: 0 = independent uniform draws (default), 1 = shuffled order
+inline uint32_t draw(int sampling, uint64_t seed, uint32_t node, int64_t n, uint64_t m) {
+    return sampling == 1 ? shuffled_index(seed, node, n, m) : sample_index(seed, node, n, m);
+}
+
 inline double widen_bf16(uint16_t b) {
     uint32_t bits = (uint32_t)b << 16;
     float f;
@@ -102,7 +148,16 @@ inline double step_size(double eta0, int sched, int64_t n) {
 
 }  // namespace
 
+static int g_sampling = 0;  // sample order used by the run functions (set by oracle_set_sampling)
+
 extern "C" {
+
+// Sample order of the run functions and of oracle_sample_indices: 0 = i.i.d. draws, 1 = shuffled order.
+int oracle_set_sampling(int mode) {
+    if (mode != 0 && mode != 1) return 1;
+    g_sampling = mode;
+    return 0;
+}
 
 // Raw generator, exposed so that tests can compare it with published vectors.
 void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
@@ -115,7 +170,7 @@ void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t
 int oracle_sample_indices(uint64_t seed, int32_t node, int64_t m, int64_t n_begin, int64_t count,
                           uint32_t* out) {
     if (m < 1 || m > 0xFFFFFFFFLL || n_begin < 0 || count < 0 || node < 0) return 1;
-    for (int64_t i = 0; i < count; ++i) out[i] = sample_index(seed, (uint32_t)node, n_begin + i + 1, (uint64_t)m);
+    for (int64_t i = 0; i < count; ++i) out[i] = draw(g_sampling, seed, (uint32_t)node, n_begin + i + 1, (uint64_t)m);
     return 0;
 }
 
@@ -134,7 +189,7 @@ int oracle_run_dense(const void* X, int xtype, int64_t ld, const float* y, const
         for (int64_t c = 0; c < d; ++c)
             w[c] = resume ? W_out[(size_t)j * d + c] : (w0 ? (double)w0[c] : 0.0);
         for (int64_t n = step_begin + 1; n <= step_begin + n_steps[j]; ++n) {
-            const int64_t row = shard_off[j] + (int64_t)sample_index(seed, (uint32_t)j, n, (uint64_t)m);
+            const int64_t row = shard_off[j] + (int64_t)draw(g_sampling, seed, (uint32_t)j, n, (uint64_t)m);
             if (xtype == 1) {
                 const uint16_t* xr = (const uint16_t*)X + (size_t)row * ld;
                 for (int64_t c = 0; c < d; ++c) x[c] = widen_bf16(xr[c]);
@@ -166,7 +221,7 @@ int oracle_run_csr_literal(const int64_t* row_ptr, const int32_t* col_idx, const
         if (n_steps[j] > 0 && m < 1) return 1;
         for (int64_t c = 0; c < d; ++c) w[c] = w0 ? (double)w0[c] : 0.0;
         for (int64_t n = 1; n <= n_steps[j]; ++n) {
-            const int64_t row = shard_off[j] + (int64_t)sample_index(seed, (uint32_t)j, n, (uint64_t)m);
+            const int64_t row = shard_off[j] + (int64_t)draw(g_sampling, seed, (uint32_t)j, n, (uint64_t)m);
             double z = 0.0;
             for (int64_t p = row_ptr[row]; p < row_ptr[row + 1]; ++p) z += w[col_idx[p]] * (double)val[p];
             const double g = loss_derivative(loss, (double)y[row], z);
@@ -195,7 +250,7 @@ int oracle_run_csr_lazy(const int64_t* row_ptr, const int32_t* col_idx, const fl
         for (int64_t c = 0; c < d; ++c) u[c] = w0 ? (double)w0[c] : 0.0;
         double s = 1.0;
         for (int64_t n = 1; n <= n_steps[j]; ++n) {
-            const int64_t row = shard_off[j] + (int64_t)sample_index(seed, (uint32_t)j, n, (uint64_t)m);
+            const int64_t row = shard_off[j] + (int64_t)draw(g_sampling, seed, (uint32_t)j, n, (uint64_t)m);
             double z = 0.0;
             for (int64_t p = row_ptr[row]; p < row_ptr[row + 1]; ++p) z += u[col_idx[p]] * (double)val[p];
             z *= s;

@@ -64,6 +64,7 @@ struct wpsgd_ctx {
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
   int opt_tc_gram = 0;
+  int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
   int opt_timing = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   bool ev_valid = false;
@@ -234,8 +235,8 @@ wpsgd_status upload_plan_and_stream(wpsgd_ctx* c, const Plan& pl) {
   CU_TRY(c, cudaMemcpyAsync(c->t_ids, c->node_ids.data(), k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   if (pl.total > 0) {
     const long long longest = *std::max_element(pl.steps.begin(), pl.steps.end());
-    dim3 grid((unsigned)grid_for((longest + 3) / 4 + 1, 256, 1024), (unsigned)std::min(k, 65535));
-    index_stream_kernel<<<grid, 256, 0, c->stream>>>(c->seed, k, c->t_idx_off, c->t_first, c->t_count, c->t_rows, c->t_ids, c->idx);
+    dim3 grid((unsigned)grid_for(c->opt_sampling ? longest + 8 : (longest + 3) / 4 + 3, 256, 1024), (unsigned)std::min(k, 65535));
+    index_stream_kernel<<<grid, 256, 0, c->stream>>>(c->opt_sampling, c->seed, k, c->t_idx_off, c->t_first, c->t_count, c->t_rows, c->t_ids, c->idx);
     CU_TRY(c, cudaGetLastError());
     c->launches++;
   }
@@ -676,6 +677,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "timing") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "timing must be 0 or 1");
     c->opt_timing = (int)value;
+  } else if (n == "sampling") {
+    if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "sampling must be 0 (i.i.d. draws) or 1 (shuffled order)");
+    c->opt_sampling = (int)value;
   } else if (n == "tc_gram") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "tc_gram must be 0 or 1");
     c->opt_tc_gram = (int)value;
@@ -849,7 +853,7 @@ wpsgd_status wpsgd_sample_indices(wpsgd_ctx* c, uint64_t seed, int32_t node, int
   if (count == 0) return WPSGD_OK;
   if (!out) return fail(c, WPSGD_ERR_INVALID_ARG, "out is NULL");
   DeviceGuard guard(c->device);
-  index_single_kernel<<<grid_for((count + 3) / 4 + 1, 256), 256, 0, c->stream>>>(seed, node, m, n_begin, count, out);
+  index_single_kernel<<<grid_for(c->opt_sampling ? count : (count + 3) / 4 + 1, 256), 256, 0, c->stream>>>(c->opt_sampling, seed, node, m, n_begin, count, out);
   CU_TRY(c, cudaGetLastError());
   c->launches++;
   return WPSGD_OK;

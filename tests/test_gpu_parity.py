@@ -68,6 +68,32 @@ def test_sample_stream_bit_exact(P, seed, node, m, n_begin, count):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("seed,node,m,n_begin,count", [
+    (0, 0, 4096, 0, 9000), (3, 7, 1, 0, 5), (3, 7, 2, 1, 9), (9, 1023, 1000, 998, 1005), (5, 2, 65537, 0, 70000),
+    (0xFFFFFFFFFFFFFFFF, 4, (1 << 32) - 1, (1 << 33) + 3, 257), (1, 1, 5, 0, 0),
+])
+def test_shuffled_sample_stream_bit_exact(P, seed, node, m, n_begin, count):
+    oracle.set_sampling(1)
+    try:
+        want = oracle.sample_indices(seed, node, m, n_begin, count)
+    finally:
+        oracle.set_sampling(0)
+    with P.Context(2, 8) as ctx:
+        ctx.set_option("sampling", 1)
+        got = ctx.sample_indices(seed, node, m, n_begin, count).cpu().numpy().view(np.uint32)
+        ctx.check()
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_small_workloads_shuffled_order(P, cfg):
+    oracle.set_sampling(1)
+    try:
+        assert_parity(P, wi.small(cfg), {"sampling": 1})
+    finally:
+        oracle.set_sampling(0)
+
+
 # ---- the five workloads, scaled down, default kernel choice ---------------------------------------------
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
 def test_small_workloads_default_kernels(P, cfg):
