@@ -162,6 +162,12 @@ wpsgd_status wpsgd_sample_indices(wpsgd_ctx* ctx, uint64_t seed, int32_t node, i
 wpsgd_status wpsgd_objective(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
                              int64_t n_rows, const float* w, float lambda, wpsgd_loss loss, double* out);
 
+/* The same two measures on CSR rows (the paper's data are sparse): row_ptr DEVICE [n_rows+1] int64, col_idx DEVICE
+ * int32 (< d), val DEVICE fp32, y DEVICE [n_rows], w DEVICE [d]; out DEVICE [2] fp64 = {objective, error}. */
+wpsgd_status wpsgd_objective_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                                 const float* y, int64_t n_rows, const float* w, float lambda, wpsgd_loss loss,
+                                 double* out);
+
 /* Whole path from HOST buffers: copies X HOST [N, d] (dense, contiguous), y HOST [N] and w0 HOST [d]
  * (or NULL) to the device, runs the chains and the combination, copies v back to v_out HOST [d], and
  * waits for completion. Page-locked host buffers give full copy speed. Device staging buffers are

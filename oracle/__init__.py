@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
             _lib.oracle_objective_dense.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, c_f32p,
                                                     ctypes.c_int64, ctypes.c_int64, c_f64p, ctypes.c_float,
                                                     ctypes.c_int, c_f64p, c_f64p]
+            _lib.oracle_objective_csr.argtypes = [c_i64p, c_i32p, c_f32p, c_f32p, ctypes.c_int64, ctypes.c_int64, c_f64p,
+                                                  ctypes.c_float, ctypes.c_int, c_f64p, c_f64p]
     return _lib
 
 
@@ -188,6 +190,15 @@ def objective_dense(X, y, w, lam, loss):
     err = np.zeros(1)
     lib().oracle_objective_dense(ptr, xtype, ld, _p(y, c_f32p), y.shape[0], w.shape[0], _p(w, c_f64p), lam, loss,
                                  _p(obj, c_f64p), _p(err, c_f64p))
+    return float(obj[0]), float(err[0])
+
+
+def objective_csr(row_ptr, col_idx, val, y, w, lam, loss):
+    rp, ci, va, y = _np(row_ptr, np.int64), _np(col_idx, np.int32), _np(val, np.float32), _np(y, np.float32)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    obj, err = np.zeros(1), np.zeros(1)
+    lib().oracle_objective_csr(_p(rp, c_i64p), _p(ci, c_i32p), _p(va, c_f32p), _p(y, c_f32p), y.shape[0], w.shape[0],
+                               _p(w, c_f64p), lam, loss, _p(obj, c_f64p), _p(err, c_f64p))
     return float(obj[0]), float(err[0])
 
 

@@ -343,4 +343,26 @@ int oracle_objective_dense(const void* X, int xtype, int64_t ld, const float* y,
     return 0;
 }
 
+// The same two measures on CSR rows.
+int oracle_objective_csr(const int64_t* row_ptr, const int32_t* col_idx, const float* val, const float* y,
+                         int64_t n_rows, int64_t d, const double* w, float lambda_f, int loss, double* objective,
+                         double* error_rate) {
+    double reg = 0.0;
+    for (int64_t c = 0; c < d; ++c) reg += w[c] * w[c];
+    double acc = 0.0;
+    int64_t wrong = 0;
+    for (int64_t i = 0; i < n_rows; ++i) {
+        double z = 0.0;
+        for (int64_t p = row_ptr[i]; p < row_ptr[i + 1]; ++p) z += w[col_idx[p]] * (double)val[p];
+        const double yy = (double)y[i];
+        if (loss == 0) acc += std::fmax(0.0, 1.0 - yy * z);
+        else if (loss == 1) acc += (yy * z > 0 ? std::log1p(std::exp(-yy * z)) : -yy * z + std::log1p(std::exp(yy * z)));
+        else acc += 0.5 * (z - yy) * (z - yy);
+        if ((z >= 0 ? 1.0 : -1.0) != (yy >= 0 ? 1.0 : -1.0)) ++wrong;
+    }
+    *objective = 0.5 * (double)lambda_f * reg + (n_rows ? acc / (double)n_rows : 0.0);
+    *error_rate = n_rows ? (double)wrong / (double)n_rows : 0.0;
+    return 0;
+}
+
 }  // extern "C"

@@ -16,7 +16,7 @@ _STATUS = {0: "OK", 1: "INVALID_ARG", 2: "ALLOC", 3: "CUDA", 4: "STATE", 5: "UNS
 EXPORTED_SYMBOLS = [
     "wpsgd_create", "wpsgd_destroy", "wpsgd_set_option", "wpsgd_set_node_ids", "wpsgd_run", "wpsgd_continue", "wpsgd_run_csr",
     "wpsgd_combine", "wpsgd_combine_weighted", "wpsgd_last_chain_ms", "wpsgd_get_models", "wpsgd_set_models", "wpsgd_get_weights", "wpsgd_weights",
-    "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_solve_host", "wpsgd_solve_static", "wpsgd_check", "wpsgd_launch_count",
+    "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_objective_csr", "wpsgd_solve_host", "wpsgd_solve_static", "wpsgd_check", "wpsgd_launch_count",
     "wpsgd_last_error",
 ]
 
@@ -64,6 +64,7 @@ def load_library() -> ctypes.CDLL:
     lib.wpsgd_weights.argtypes = [vp, i32, f32, ci, f32, f64, vp, ctypes.POINTER(ci), ctypes.POINTER(f64)]
     lib.wpsgd_sample_indices.argtypes = [vp, u64, i32, i64, i64, i64, vp]
     lib.wpsgd_objective.argtypes = [vp, vp, ci, i64, vp, i64, vp, f32, ci, vp]
+    lib.wpsgd_objective_csr.argtypes = [vp, vp, vp, vp, vp, i64, vp, f32, ci, vp]
     lib.wpsgd_solve_host.argtypes = [vp, vp, ci, vp, vp, vp, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_solve_static.argtypes = [ci, vp, vp, ci, i64, vp, vp, vp, i32, i64, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_check.argtypes = [vp]
@@ -311,6 +312,17 @@ class Context:
                                            self._dev(y, torch.float32, X.shape[0]), X.shape[0],
                                            self._dev(w, torch.float32, self.d), lam, loss, self._dev(out)),
                  "wpsgd_objective")
+        return out
+
+    def objective_csr(self, row_ptr, col_idx, val, y, w, lam: float, loss: int):
+        import torch
+
+        out = torch.empty(2, dtype=torch.float64, device=f"cuda:{self.device}")
+        n_rows = int(y.numel())
+        self._ck(self._lib.wpsgd_objective_csr(self._h, self._dev(row_ptr, torch.int64, n_rows + 1),
+                                               self._dev(col_idx, torch.int32), self._dev(val, torch.float32),
+                                               self._dev(y, torch.float32), n_rows, self._dev(w, torch.float32, self.d),
+                                               lam, loss, self._dev(out)), "wpsgd_objective_csr")
         return out
 
     def solve_host(self, X, y, shard_off, n_steps, eta0, sched, lam, loss, seed, w0=None, r: float = 0.0, out=None):

@@ -79,6 +79,41 @@ __global__ void __launch_bounds__(256) objective_rows_kernel(const XT* __restric
   }
 }
 
+// Pass 1 on CSR rows: one warp per row, lanes over the row's nonzeros.
+__global__ void __launch_bounds__(256) objective_rows_csr_kernel(const long long* __restrict__ row_ptr,
+                                                                 const int* __restrict__ col_idx,
+                                                                 const float* __restrict__ val,
+                                                                 const float* __restrict__ y, long long n_rows,
+                                                                 const float* __restrict__ w, int loss,
+                                                                 double* __restrict__ part) {
+  __shared__ double sl[8], se[8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double lsum = 0.0, esum = 0.0;
+  for (long long i = (long long)blockIdx.x * 8 + warp; i < n_rows; i += (long long)gridDim.x * 8) {
+    const long long b = row_ptr[i], e = row_ptr[i + 1];
+    float acc = 0.0f;
+    for (long long q = b + lane; q < e; q += 32) acc = fmaf(w[col_idx[q]], val[q], acc);
+    const float z = warp_sum(acc);
+    const float yy = y[i];
+    double L;
+    if (loss == LOSS_HINGE) L = fmax(0.0, 1.0 - (double)yy * (double)z);
+    else if (loss == LOSS_LOGISTIC) {
+      const double t = (double)yy * (double)z;
+      L = t > 0 ? log1p(exp(-t)) : -t + log1p(exp(t));
+    } else L = 0.5 * ((double)z - (double)yy) * ((double)z - (double)yy);
+    lsum += L;
+    esum += ((z >= 0.0f) != (yy >= 0.0f)) ? 1.0 : 0.0;
+  }
+  if (lane == 0) { sl[warp] = lsum; se[warp] = esum; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0, b2 = 0.0;
+    for (int i = 0; i < 8; ++i) { a += sl[i]; b2 += se[i]; }
+    part[2 * blockIdx.x] = a;
+    part[2 * blockIdx.x + 1] = b2;
+  }
+}
+
 // Pass 2: out[0] = (lambda/2)|w|^2 + sum(part loss)/n_rows, out[1] = sum(part err)/n_rows. One block.
 __global__ void __launch_bounds__(256) objective_finish_kernel(const double* __restrict__ part, int n_part,
                                                                const float* __restrict__ w, long long d, float lambda,

@@ -880,6 +880,25 @@ wpsgd_status wpsgd_objective(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, int64_
   return WPSGD_OK;
 }
 
+wpsgd_status wpsgd_objective_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                                 const float* y, int64_t n_rows, const float* w, float lambda, wpsgd_loss loss,
+                                 double* out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!w || !out || n_rows < 0 || (int)loss < 0 || (int)loss > 2 || (n_rows > 0 && (!row_ptr || !col_idx || !val || !y)))
+    return fail(c, WPSGD_ERR_INVALID_ARG, "objective_csr: bad argument");
+  DeviceGuard guard(c->device);
+  const int nblk = grid_for((n_rows + 7) / 8, 1, 148 * 8);
+  wpsgd_status s = grow(c, &c->part, &c->part_cap, (size_t)nblk * 2);
+  if (s != WPSGD_OK) return s;
+  objective_rows_csr_kernel<<<nblk, 256, 0, c->stream>>>((const long long*)row_ptr, col_idx, val, y, n_rows, w, (int)loss,
+                                                         c->part);
+  CU_TRY(c, cudaGetLastError());
+  objective_finish_kernel<<<1, 256, 0, c->stream>>>(c->part, nblk, w, c->d, lambda, n_rows, out);
+  CU_TRY(c, cudaGetLastError());
+  c->launches += 2;
+  return WPSGD_OK;
+}
+
 wpsgd_status wpsgd_solve_host(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, const float* y, const int64_t* shard_off,
                               const int64_t* n_steps, float eta0, wpsgd_lr sched, float lambda, wpsgd_loss loss,
                               uint64_t seed, const float* w0, double r, float* v_out) {

@@ -403,3 +403,22 @@ def test_objective_and_error_rate_by_hand():
     obj, _ = oracle.objective_dense(X, y, w, f32(0.0), LOGISTIC)
     assert obj == pytest.approx((np.log1p(np.exp(-0.5)) + np.log1p(np.exp(0.5)) + np.log1p(np.exp(-0.75))) / 3,
                                 rel=1e-14)
+
+
+def test_csr_objective_by_hand_and_against_dense():
+    # rows: [1, 0], [0, 2], [1, 1] as CSR; same numbers as the dense hand example above
+    rp = np.array([0, 1, 2, 4], dtype=np.int64)
+    ci = np.array([0, 1, 0, 1], dtype=np.int32)
+    va = np.array([1.0, 2.0, 1.0, 1.0], dtype=np.float32)
+    y = np.array([1.0, -1.0, 1.0], dtype=np.float32)
+    w = np.array([0.5, 0.25])
+    obj, err = oracle.objective_csr(rp, ci, va, y, w, f32(0.5), HINGE)
+    assert obj == pytest.approx(0.75 + 0.5 * 0.5 * 0.3125, rel=1e-14)
+    assert err == pytest.approx(1.0 / 3.0)
+    wl = _small_sparse()
+    dn = wi.densify(wl)
+    wv = np.random.default_rng(0).normal(size=wl.d)
+    for loss in (HINGE, LOGISTIC, SQUARED):
+        a = oracle.objective_csr(wl.row_ptr, wl.col_idx, wl.val, wl.y, wv, f32(0.1), loss)
+        b = oracle.objective_dense(dn.X, dn.y, wv, f32(0.1), loss)
+        assert a[0] == pytest.approx(b[0], rel=1e-12) and a[1] == b[1]
