@@ -97,6 +97,16 @@ def weights(n_steps, eta0: float, sched: int, lam: float, r: float = 0.0) -> Tup
     return w, bool(flag.value), float(tot.value)
 
 
+def averaging_span_valid(n_steps, eta0: float, lam: float, span: int, r: float = 0.0) -> Tuple[bool, float]:
+    """Condition the paper gives for averaging every `span` fastest-node steps on an unbalanced system
+    (Section "Combining WP-SGD with bucket SGD"): (k / sum_j r^{T_j}) * (1 - eta lambda)^span < 1.
+    Returns (holds, left-hand side); sum_j r^{T_j} comes from wpsgd_weights."""
+    n = _host_i64(n_steps)
+    _, _, tot = weights(n, eta0, LR_CONST, lam, r)
+    lhs = (n.shape[0] / tot) * (1.0 - float(np.float32(eta0)) * float(np.float32(lam))) ** int(span)
+    return bool(lhs < 1.0), float(lhs)
+
+
 def _xtype(X) -> int:
     import torch
 

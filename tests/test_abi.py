@@ -98,3 +98,19 @@ def test_create_without_device_reports_error_instead_of_crashing(wpsgd_lib):
     assert wpsgd_lib.wpsgd_create(0, None, 0, 64, ctypes.byref(h)) == 1
     assert wpsgd_lib.wpsgd_destroy(None) == 0
     assert wpsgd_lib.wpsgd_check(None) == 1
+
+
+def test_validity_condition_of_averaging_every_span(wpsgd_lib):
+    import paper_1708_04801_b200 as P
+
+    # k = 4, delays 0, 0, 1000, 1000 at r = 1 - 0.1 * 0.01 = 0.999: sum r^T = 2 + 2 * 0.999^1000
+    n = [2000, 2000, 1000, 1000]
+    r = 1.0 - float(np.float32(0.1)) * float(np.float32(0.01))
+    tot = 2 + 2 * r ** 1000
+    for span, want in ((100, (4 / tot) * r ** 100), (1000, (4 / tot) * r ** 1000)):
+        holds, lhs = P.averaging_span_valid(n, 0.1, 0.01, span)
+        assert lhs == pytest.approx(want, rel=1e-9)
+        assert holds == (want < 1.0)
+    assert P.averaging_span_valid(n, 0.1, 0.01, 100)[0] is False   # a short span cannot make up for the delays
+    assert P.averaging_span_valid(n, 0.1, 0.01, 1000)[0] is True
+    assert P.averaging_span_valid([50, 50, 50], 0.1, 0.01, 1)[0] is True   # balanced: any span is valid
