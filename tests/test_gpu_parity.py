@@ -476,3 +476,42 @@ def test_errors_are_reported_not_thrown_from_c(P):
         ctx.combine()
         ctx.check()
         assert ctx.launch_count() >= 3
+
+
+# ---- shapes at the edges of the launch configurations ---------------------------------------------------------------
+def test_many_nodes_with_few_steps(P):
+    k, d, m = 3000, 64, 4
+    g = torch.Generator().manual_seed(11)
+    X = torch.randn(k * m, d, generator=g) / 8
+    y = torch.sign(torch.randn(k * m, generator=g))
+    n = (np.arange(k) % 7).astype(np.int64)  # 0..6 steps, many idle nodes, ragged last CTA
+    wl = wi.Workload("many", k, d, np.arange(k + 1, dtype=np.int64) * m, n, 0.05, 0, 0.01, LOGISTIC, 5, y, X=X)
+    assert_parity(P, wl)
+    assert_parity(P, wl, {"dense_variant": 3})
+
+
+@pytest.mark.parametrize("d", [1, 2, 3, 5])
+def test_tiny_feature_counts(P, d):
+    g = torch.Generator().manual_seed(d)
+    k, m = 3, 20
+    X = torch.randn(k * m, d, generator=g)
+    y = torch.sign(torch.randn(k * m, generator=g))
+    wl = wi.Workload("tiny", k, d, np.arange(k + 1, dtype=np.int64) * m, np.array([60, 1, 33]), 0.05, 0, 0.01, LOGISTIC, 3,
+                     y, X=X)
+    assert_parity(P, wl)
+
+
+def test_one_long_chain(P):
+    wl = wi.config2(k=1, d=256, m=512, base_steps=60000)
+    assert_parity(P, wl)
+
+
+def test_csr_rows_without_nonzeros_and_single_nonzero(P):
+    # hand-built CSR: rows 0 and 3 are empty, row 1 has one nonzero, row 2 three
+    rp = torch.tensor([0, 0, 1, 4, 4, 6], dtype=torch.int64)
+    ci = torch.tensor([5, 0, 3, 7, 1, 6], dtype=torch.int32)
+    va = torch.tensor([2.0, 0.5, -1.0, 0.25, 1.5, -0.75])
+    y = torch.tensor([1.0, -1.0, 1.0, -1.0, 1.0])
+    wl = wi.Workload("gaps", 1, 8, np.array([0, 5]), np.array([200]), 0.1, 1, 0.05, LOGISTIC, 2, y, row_ptr=rp, col_idx=ci,
+                     val=va, w0=torch.full((8,), 0.3))
+    assert_parity(P, wl)
