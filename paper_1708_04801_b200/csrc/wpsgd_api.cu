@@ -12,6 +12,7 @@
 
 #include "chain_block.cuh"
 #include "chain_csr.cuh"
+#include "chain_tc.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
 #include "philox.cuh"
@@ -208,9 +209,9 @@ wpsgd_status make_plan(wpsgd_ctx* c, const long long* shard_off, const long long
     if (n_steps[j] > 0 && m < 1) return fail(c, WPSGD_ERR_INVALID_ARG, "a node with steps has an empty shard");
     if (m > 0xFFFFFFFFll) return fail(c, WPSGD_ERR_INVALID_ARG, "a shard has 2^32 rows or more");
     pl->rows[j] = m;
-    // the stream of a node is produced up to the next multiple of 8 steps (the draws simply continue), so
-    // that kernels that take samples in groups always read valid rows
-    pl->count[j] = (n_steps[j] + 7) / 8 * 8;
+    // the stream of a node is produced up to the next multiple of 64 steps (the draws simply continue), so
+    // that kernels that take samples in groups of 8 or 64 always read valid rows
+    pl->count[j] = (n_steps[j] + 63) / 64 * 64;
     pl->idx_off[j + 1] = pl->idx_off[j] + pl->count[j];
   }
   pl->total = pl->idx_off[k];
@@ -368,6 +369,51 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
               : launch_block_r<XT, 2, false, 8, false>(c, bp, threads, smem);
 }
 
+// ---- blocked kernel with the Gram products on tcgen05 (bf16 rows) --------------------------------------------------
+bool tc_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out) {
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  if (c->d % 64 != 0) return false;
+  const long long chunks = c->d / 8;
+  const int R = (int)((chunks + 32 * TC_MATH_WARPS - 1) / (32 * TC_MATH_WARPS));
+  if (R > 2) return false;
+  const size_t row_bytes = (size_t)c->d * 2 + 16;
+  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 3;
+  while (stages >= 2 && TcSmem(stages, row_bytes).total > kSmemBudget) --stages;
+  if (stages < 2) return false;
+  *R_out = R;
+  *stages_out = stages;
+  return true;
+}
+
+template <int R>
+wpsgd_status launch_tc_r(wpsgd_ctx* c, const BlockParams& bp, size_t smem) {
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<c->k, TC_THREADS, smem, c->stream>>>(bp);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_tc_kernel<R, LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_tc_kernel<R, LOSS_LOGISTIC>);
+    default: return go(chain_tc_kernel<R, LOSS_SQUARED>);
+  }
+}
+
+wpsgd_status launch_tc(wpsgd_ctx* c, const ChainParams& p, int R, int stages) {
+  BlockParams bp;
+  bp.c = p;
+  bp.stages = stages;
+  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  bp.spin_limit = c->opt_spin_limit;
+  bp.drop_block = c->opt_drop_block;
+  bp.group_order = nullptr;
+  const size_t smem = TcSmem(stages, (size_t)c->d * 2 + 16).total;
+  return R == 1 ? launch_tc_r<1>(c, bp, smem) : launch_tc_r<2>(c, bp, smem);
+}
+
 // blocked kernel, one warp per node (small d)
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
@@ -465,6 +511,14 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
   }
+  if (variant == 6 || (variant == 4 && c->opt_tc_gram == 2)) {
+    int tR = 0, tstages = 0;
+    if (sizeof(XT) != 2 || !tc_kernel_fits(c, aligned, &tR, &tstages))
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "tcgen05 kernel needs bf16 rows, 16-byte aligned, d a multiple of 64 and at most 4096, a constant "
+                  "step size and eta*lambda <= 0.25");
+    return launch_tc(c, p, tR, tstages);
+  }
   if (variant == 4) {
     if (!block_ok)
       return fail(c, WPSGD_ERR_UNSUPPORTED,
@@ -541,7 +595,7 @@ constexpr size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 struct StaticLayout {
   size_t W = 0;
   size_t idx = align256(W + sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS);
-  size_t shard_off = align256(idx + sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES));
+  size_t shard_off = align256(idx + sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 64 * WPSGD_STATIC_MAX_NODES));
   size_t steps = align256(shard_off + sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
   size_t first = align256(steps + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
   size_t idx_off = align256(first + sizeof(long long) * WPSGD_STATIC_MAX_NODES);
@@ -556,7 +610,7 @@ struct StaticLayout {
   size_t total = align256(status + sizeof(DevStatus));
 };
 constexpr size_t kStaticBytes = align256(sizeof(float) * (size_t)WPSGD_STATIC_MAX_MODEL_ELEMS) +
-                                align256(sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES)) +
+                                align256(sizeof(uint32_t) * ((size_t)WPSGD_STATIC_MAX_STEPS + 64 * WPSGD_STATIC_MAX_NODES)) +
                                 13 * align256(sizeof(long long) * (WPSGD_STATIC_MAX_NODES + 1));
 constexpr int kStaticMaxDevices = 64;
 }  // namespace
@@ -654,7 +708,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 5) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..5");
+    if (value < 0 || value > 6) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..6");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");
@@ -681,7 +735,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "sampling must be 0 (i.i.d. draws) or 1 (shuffled order)");
     c->opt_sampling = (int)value;
   } else if (n == "tc_gram") {
-    if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "tc_gram must be 0 or 1");
+    if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "tc_gram must be 0, 1 or 2");
     c->opt_tc_gram = (int)value;
   } else if (n == "test_drop_block") {
     c->opt_drop_block = value;
@@ -984,7 +1038,7 @@ wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wp
   const StaticLayout L;
   c.W = (float*)(base + L.W);
   c.idx = (uint32_t*)(base + L.idx);
-  c.idx_cap = (size_t)WPSGD_STATIC_MAX_STEPS + 8 * WPSGD_STATIC_MAX_NODES;  // never regrown: padding included
+  c.idx_cap = (size_t)WPSGD_STATIC_MAX_STEPS + 64 * WPSGD_STATIC_MAX_NODES;  // never regrown: padding included
   c.t_shard_off = (long long*)(base + L.shard_off);
   c.t_steps = (long long*)(base + L.steps);
   c.t_first = (long long*)(base + L.first);

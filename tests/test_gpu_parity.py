@@ -229,6 +229,37 @@ def test_bounded_wait_for_rows_reports_timeout_and_context_survives(P, d, bf16):
     assert rel_l2(v, ov) <= 1e-4
 
 
+# ---- tcgen05 kernel: Gram blocks of 64 samples at a time on the tensor cores (bf16 rows) ---------------------------
+@pytest.mark.parametrize("n_steps", [(1, 63, 64), (65, 127, 128), (129, 0, 200), (700, 333, 8)])
+@pytest.mark.parametrize("d", [64, 512, 1024, 4096])
+def test_tcgen05_kernel_superblock_boundaries(P, n_steps, d):
+    wl = wi.config3(k=3, d=d, m=96, n_lo=10, n_hi=20)
+    wl.n_steps = np.array(n_steps, dtype=np.int64)
+    wl.w0 = torch.full((d,), 0.05)
+    assert_parity(P, wl, {"dense_variant": 6})
+
+
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("stages", [2, 3])
+def test_tcgen05_kernel_losses_and_ring_depths(P, loss, stages):
+    wl = wi.config2(k=5, d=2048, m=80, base_steps=300)
+    wl.X = wl.X.to(torch.bfloat16)
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    assert_parity(P, wl, {"dense_variant": 6, "stages": stages})
+
+
+def test_tcgen05_kernel_limits(P):
+    wl = wi.config2(k=2, d=1024, m=16, base_steps=20)  # fp32 rows
+    with pytest.raises(P.WpsgdError) as e:
+        gpu_solve(P, wl, {"dense_variant": 6})
+    assert e.value.status_name == "UNSUPPORTED"
+    wl = wi.config3(k=2, d=4096 + 8, m=16, n_lo=10, n_hi=20)  # d not a multiple of 64
+    with pytest.raises(P.WpsgdError):
+        gpu_solve(P, wl, {"dense_variant": 6})
+
+
 def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
     wl = wi.config2(k=4, d=1024, m=64, base_steps=100).to("cuda")
     with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
