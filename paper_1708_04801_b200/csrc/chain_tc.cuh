@@ -27,7 +27,9 @@
 namespace wpsgd {
 
 constexpr int TC_SB = 64;        // samples per super-block (rows of one tcgen05 product)
-constexpr int TC_NB = 6;         // tile buffers of the Gram stream
+constexpr int TC_NB = 10;        // tile buffers of the Gram stream
+constexpr int TC_D = 7;          // copies run TC_D - 1 chunks ahead of the multiply; a buffer is refilled TC_NB - TC_D + 1
+                                 // chunks after the multiply that read it was issued, so that wait is never on the path
 constexpr int TC_TILE = 8192;    // bytes of a tile: 64 rows x 64 bf16 columns
 constexpr int TC_MATH_WARPS = 8;
 constexpr int TC_THREADS = 32 * (6 + TC_MATH_WARPS);
@@ -284,36 +286,49 @@ __global__ void __launch_bounds__(TC_THREADS, 1) chain_tc_kernel(const BlockPara
   if (warp < 6) {
     // =========================== Gram warps ================================================================
     const int gt = threadIdx.x - 64;   // 0..127
-    const int row = gt & 63;           // row of the super-block this thread copies
-    const int c0 = gt >> 6;            // it copies 16-byte chunks c0, c0+2, c0+4, c0+6 of every 128-byte row segment
+    const int wq = gt >> 5;            // Gram warp number 0..3
+    // Copy assignment: a warp instruction moves 8 rows x 64 contiguous bytes (lane -> row lane & 7, 16-byte chunk
+    // lane >> 3 of the half), so global reads are whole sectors of 8 lines and the shared-memory writes of a
+    // warp fall on 8 different 16-byte bank groups in each of 4 chunk planes (no conflicts). Over its 4 copies
+    // per tile a thread covers two rows, 8 (2 wq) + rr and 8 (2 wq + 1) + rr, both halves of each.
+    const int rr = lane & 7, cc = lane >> 3;
     const int q = warp & 3;            // tensor-memory subpartition this warp can read: rows 16q .. 16q+15
     const uint32_t tmem = *tmem_holder;
     const long long total = nsb * CK;  // 64-column chunks over the whole chain
     // producer position (chunk being copied) and consumer position (chunk being multiplied)
-    long long gi = 0; int kci = 0; long long si = 0; const char* rowptr = nullptr; long long row_sb = -1;
+    long long gi = 0; int kci = 0; long long si = 0; long long row_sb = -1;
+    const char* rowptr[2] = {nullptr, nullptr};
     bool failed = false;
     auto issue_copy = [&]() {  // copy this thread's part of chunk gi into tile buffer gi % TC_NB; one group per call
       if (gi < total) {
         if (row_sb != si) {
-          rowptr = shard + (size_t)idx[si * TC_SB + row] * ld_bytes;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int row = 8 * (2 * wq + h) + rr;
+            rowptr[h] = shard + (size_t)idx[si * TC_SB + row] * ld_bytes;
+            if (cc == 0 && si + 1 < nsb) {  // ask L2 for the same row slot of the next super-block
+              const char* nxt = shard + (size_t)idx[(si + 1) * TC_SB + row] * ld_bytes;
+              asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(nxt), "r"((uint32_t)(d * sizeof(XT))) : "memory");
+            }
+          }
           row_sb = si;
         }
         unsigned char* tile = tiles + (size_t)(gi % TC_NB) * TC_TILE;
-        const char* src = rowptr + (size_t)kci * 128;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int c = c0 + 2 * i;
-          cp_async16(tile + c * 1024 + row * 16, src + c * 16);
+          const int h = i >> 1, half = i & 1;         // row group 2 wq + h, chunks 4 half + cc
+          const int row = 8 * (2 * wq + h) + rr, c = 4 * half + cc;
+          cp_async16(tile + c * 1024 + row * 16, rowptr[h] + (size_t)kci * 128 + c * 16);
         }
         ++gi;
         if (++kci == CK) { kci = 0; ++si; }
       }
       cp_async_commit();
     };
-    for (int i = 0; i < TC_NB - 1; ++i) issue_copy();
+    for (int i = 0; i < TC_D - 1; ++i) issue_copy();
     int kc = 0; long long s = 0;
     for (long long g = 0; g < total; ++g) {
-      cp_async_wait(TC_NB - 2);  // this thread's part of chunk g has landed (TC_NB - 1 + g groups committed)
+      cp_async_wait(TC_D - 2);  // this thread's part of chunk g has landed (TC_D - 1 + g groups committed)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       // all 128 parts of the tile are in place; the same barrier carries the decision to stop
       if (named_sync_or(3, 128, failed || *chain_over != 0)) break;
@@ -330,10 +345,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) chain_tc_kernel(const BlockPara
         umma_commit(&mma_bars[u]);                    // the tile may be refilled once these have read it
         if (kc == CK - 1) umma_commit(&sb_bars[s & 1]);  // the super-block's product is complete
       }
-      // refill the buffer of chunk g-1 with chunk g + TC_NB - 1 once the tensor core has read it
-      if (g >= 1 && gi < total) {
-        const int up = (int)((g - 1) % TC_NB);
-        if (!mbar_wait_bounded(&mma_bars[up], (uint32_t)(((g - 1) / TC_NB) & 1), bp.spin_limit)) failed = true;
+      // chunk g + TC_D - 1 goes into the buffer last read by the multiply of chunk g + TC_D - 1 - TC_NB
+      if (g + TC_D - 1 >= TC_NB && gi < total) {
+        const long long old = g + TC_D - 1 - TC_NB;
+        if (!mbar_wait_bounded(&mma_bars[old % TC_NB], (uint32_t)((old / TC_NB) & 1), bp.spin_limit)) failed = true;
       }
       issue_copy();
       if (kc == CK - 1) {
