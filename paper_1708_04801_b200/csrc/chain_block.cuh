@@ -151,6 +151,38 @@ __device__ __forceinline__ float warp_transpose_sum8(float (&v)[8]) {
   return t;
 }
 
+// Logistic loss in the blocked recurrence. With t the margin times y log2(e), the step needs s(t) = 1 / (1 + 2^t):
+// two special-function evaluations in the dependent chain of every sample. Inside a block the argument of sample n is
+// t0_n + delta_n, where t0_n (from p_n) is known before the recurrence starts and delta_n collects the block's earlier
+// steps. s and its first three derivatives at t0_n are formed for all samples of the block at once; the chain then
+// only evaluates a cubic in delta_n. Remainder: |d4s/dt4| delta^4 / 24 < 2e-8 for |delta| < 1/16; a block in which
+// some delta is larger is run again with the direct evaluation (kept out of the fast loop, so that no
+// special-function unit sits in its dependent chain).
+constexpr float LOGISTIC_DELTA_MAX = 0.0625f;
+__device__ __forceinline__ float logistic_factor(float t) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return r;
+}
+// (s, ds/dt, d2s/dt2 / 2, d3s/dt3 / 6) at t0. With x = t ln2 and f = 1/(1+e^x): df = -f(1-f), d2f = f(1-f)(1-2f),
+// d3f = f(1-f)(6f(1-f) - 1).
+__device__ __forceinline__ float4 logistic_jet(float t0) {
+  constexpr float q = 0.6931471805599453f;
+  const float f = logistic_factor(t0);
+  const float h = f * (1.0f - f);
+  float4 j;
+  j.x = f;
+  j.y = -q * h;
+  j.z = (0.5f * q * q) * h * fmaf(-2.0f, f, 1.0f);
+  j.w = (q * q * q / 6.0f) * h * fmaf(6.0f, h, -1.0f);
+  return j;
+}
+// The cubic at delta (valid while |delta| < LOGISTIC_DELTA_MAX).
+__device__ __forceinline__ float logistic_factor_near(const float4& jet, float delta) {
+  return fmaf(delta, fmaf(delta, fmaf(delta, jet.w, jet.z), jet.y), jet.x);
+}
+
 // 8x8 b16 tiles from shared memory, four at a time (lanes 8i..8i+7 give the row addresses of tile i); each
 // lane receives, per tile, the pair of elements (row = lane / 4, columns 2 (lane % 4), +1).
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_ptr) {
@@ -175,7 +207,7 @@ constexpr int BLK_MAX_MATH_WARPS = 16;
 
 // Shared-memory carve-up (bytes). Ring first (16-byte aligned), then the small arrays.
 struct BlockSmem {
-  size_t ring, redG, redP, totG, gam, tab, bars, flag, total;
+  size_t ring, redG, redP, totG, gam, tab, jet, bars, flag, total;
   __host__ __device__ BlockSmem(int stages, size_t row_bytes, int math_warps) {
     ring = 0;
     redG = ring + (size_t)stages * BLK_B * row_bytes;
@@ -184,7 +216,8 @@ struct BlockSmem {
     totG = redP + (size_t)BLK_MAX_MATH_WARPS * BLK_B * sizeof(float);
     gam = totG + 64 * sizeof(float);
     tab = gam + 16 * sizeof(float);
-    bars = (tab + 3 * 16 * sizeof(float) + 7) / 8 * 8;  // one arrival barrier per ring stage (up to 8)
+    jet = tab + 3 * 16 * sizeof(float);  // 8 x (s, s', s''/2, s'''/6) of the logistic factor
+    bars = jet + 8 * 4 * sizeof(float);  // one arrival barrier per ring stage (up to 8)
     flag = bars + 8 * sizeof(unsigned long long);
     total = flag + 16;
   }
@@ -217,6 +250,7 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
   float* totG = (float*)(smem + L.totG);   // [32] Gram entries summed over the math warps
   float* gam = (float*)(smem + L.gam);     // gamma_0..7, [8] = 1 - a^nv
   float* tab = (float*)(smem + L.tab);     // [0..8] a^k, [16..24] eta / a^{k+1}, [32..40] 1 - a^k
+  float4* jets = (float4*)(smem + L.jet);  // logistic factor and derivatives of the block's 8 samples
   unsigned long long* bars = (unsigned long long*)(smem + L.bars);  // bars[s]: rows of the block in stage s have landed
   volatile int* give_up = (volatile int*)(smem + L.flag);           // set when a bounded wait ran out
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes;
@@ -342,20 +376,54 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
+      if (LOSS == LOSS_LOGISTIC) {
+        // lane n & 7 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
+        if (lane < B) jets[lane] = logistic_jet(y_cur * tab[n] * 1.4426950408889634f * psum);
+        __syncwarp();
+        float4 jet[B];
+        float dlt[B];
 #pragma unroll
-      for (int m = 0; m < B; ++m) {
-        if (LOSS == LOSS_LOGISTIC) {
-          float e, r;
-          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t[m]));
-          asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
-          beta[m] = cf[m] * r;
-        } else if (LOSS == LOSS_HINGE) {
-          beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
-        } else {
-          beta[m] = cf[m] * (t[m] - yv[m]);
+        for (int m = 0; m < B; ++m) {
+          jet[m] = jets[m];
+          dlt[m] = 0.0f;
         }
+        float dmax = 0.0f;
 #pragma unroll
-        for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+        for (int m = 0; m < B; ++m) {
+          dmax = fmaxf(dmax, fabsf(dlt[m]));
+          beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
+#pragma unroll
+          for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
+        }
+        if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
+#pragma unroll 1
+          for (int m = 0; m < B; ++m) {
+            float tm_ = 0.0f, cfm = 0.0f;
+#pragma unroll
+            for (int q = 0; q < B; ++q)
+              if (q == m) { tm_ = t[q]; cfm = cf[q]; }
+            const float bm = cfm * logistic_factor(tm_);
+#pragma unroll
+            for (int q = 0; q < B; ++q)
+              if (q == m) beta[q] = bm;
+#pragma unroll
+            for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+              for (int q = 0; q < n2; ++q)
+                if (q == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + q], t[n2]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int m = 0; m < B; ++m) {
+          if (LOSS == LOSS_HINGE) {
+            beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+          } else {
+            beta[m] = cf[m] * (t[m] - yv[m]);
+          }
+#pragma unroll
+          for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+        }
       }
       // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}
       float mine = dl_nv;
@@ -823,20 +891,58 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
 #pragma unroll
       for (int k2 = 0; k2 < m; ++k2) Gs[m * (m - 1) / 2 + k2] *= sc;
     }
+    if (LOSS == LOSS_LOGISTIC) {
+      // lane n & 7 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
+      // through the warp's scratch line (its Gram entries and p are in registers by now)
+      const float t_own = y_cur * tab[n] * 1.4426950408889634f * scratch[32 + n];
+      __syncwarp();
+      if (lane < B) ((float4*)scratch)[lane] = logistic_jet(t_own);
+      __syncwarp();
+      float4 jet[B];
+      float dlt[B];
 #pragma unroll
-    for (int m = 0; m < B; ++m) {
-      if (LOSS == LOSS_LOGISTIC) {
-        float e, r;
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t[m]));
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
-        beta[m] = cf[m] * r;
-      } else if (LOSS == LOSS_HINGE) {
-        beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
-      } else {
-        beta[m] = cf[m] * (t[m] - yv[m]);
+      for (int m = 0; m < B; ++m) {
+        jet[m] = ((const float4*)scratch)[m];
+        dlt[m] = 0.0f;
       }
+      __syncwarp();
+      float dmax = 0.0f;
 #pragma unroll
-      for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+      for (int m = 0; m < B; ++m) {
+        dmax = fmaxf(dmax, fabsf(dlt[m]));
+        beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
+#pragma unroll
+        for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
+      }
+      if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
+#pragma unroll 1
+        for (int m = 0; m < B; ++m) {
+          float tm_ = 0.0f, cfm = 0.0f;
+#pragma unroll
+          for (int q = 0; q < B; ++q)
+            if (q == m) { tm_ = t[q]; cfm = cf[q]; }
+          const float bm = cfm * logistic_factor(tm_);
+#pragma unroll
+          for (int q = 0; q < B; ++q)
+            if (q == m) beta[q] = bm;
+#pragma unroll
+          for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+            for (int q = 0; q < n2; ++q)
+              if (q == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + q], t[n2]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        if (LOSS == LOSS_HINGE) {
+          beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+        } else {
+          beta[m] = cf[m] * (t[m] - yv[m]);
+        }
+#pragma unroll
+        for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+      }
     }
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m,  gamma_m = beta_m a^nv ----------------------------------
 #pragma unroll

@@ -1,0 +1,474 @@
+// Per-node SGD chains on dense bf16 rows, blocked form (see chain_block.cuh for the algebra), with the Gram block
+// and the margins of a block from the warp-level tensor-core instruction and the columns of a chain split over the
+// CTAs of a thread-block cluster.
+//
+// What a block of B = 8 samples needs before its scalar recurrence is G = X_b X_b^T (8 x 8) and p = X_b w (8): one
+// product [X_b ; w] X_b^T of an (8 + 1) x d by a d x 8 matrix. The rows are bf16, so their products are exact in fp32
+// and the tensor core accumulates them in fp32. The model is fp32; it is written as w = w_hi + w_mid + w_lo with three
+// bf16 terms (8 + 8 + 8 mantissa bits, each remainder exact), which enter the product as three more rows. One
+// mma.m16n8k16 per 16 columns then gives, in its 16 x 8 accumulator, rows 0..7 = G and rows 8..10 = the three parts
+// of p: no widening of the rows, no FMA per column pair, no cross-lane reduction (the instruction sums over its 16
+// columns, the accumulator over the warp's 256). Only the update w <- w - (1 - a^B) w - sum_m gamma_m x_m stays on
+// the fp32 pipes (packed two-wide FMAs), followed by re-splitting the thread's 8 model values into the three bf16 rows.
+//
+// Layout. CTA `rank` of a cluster of C owns the 16-byte chunks [rank * cpc, (rank + 1) * cpc) of every row; math warp
+// mw owns chunks [32 mw, 32 mw + 32) of that slice, lane l chunk 32 mw + l (its 8 model values live in registers).
+// Warp 0 runs the recurrence, warp 1 requests rows (bulk asynchronous copies into a ring of stages, one barrier per
+// stage, never multicast). Staged rows and the three model rows have a stride of slice + 16 bytes, which keeps the
+// 8 x 8 tile loads (ldmatrix) free of bank conflicts; bytes beyond a CTA's slice stay zero.
+//
+// Exchange inside the cluster. Every math warp sends its 64 + 24 accumulator values to the partial-sum table of
+// every CTA of the cluster with st.async (a store to distributed shared memory that reports its bytes to a barrier
+// of the destination CTA). The recurrence warp of each CTA arms that barrier with the byte count of all math warps
+// of the cluster and waits for it (bounded), adds the partial sums, runs the recurrence and publishes gamma in its
+// own CTA: every CTA does this redundantly, so there is one exchange per block and no cluster-wide barrier inside
+// the loop. Tables and barriers are double buffered by block parity; a CTA cannot receive block b + 2 before it has
+// consumed block b, because its peers need its own block b + 1 first.
+//
+// Leaving. A wait that runs out (rows or partial sums) sets the status word and the give-up flag of every CTA of
+// the cluster. The recurrence warp samples the flag once per block and publishes the decision with gamma, so all
+// warps of a CTA leave at the same block; every thread then passes one final cluster barrier, so no CTA exits while
+// a peer may still store into its shared memory.
+#pragma once
+
+#include "chain_cluster.cuh"
+
+namespace wpsgd {
+
+constexpr int MMA_SLOTS = 16;    // math warps of a whole cluster
+constexpr int MMA_G_VALS = 64;   // accumulator rows 0..7
+constexpr int MMA_P_VALS = 32;   // accumulator rows 8..10 (24 used)
+constexpr uint32_t MMA_SLOT_BYTES = (64 + 24) * sizeof(float);  // what one math warp sends to one CTA per block
+
+struct MmaSmem {
+  size_t row_stride, ring, w3, redG, redP, totG, gam, tab, jet, bars, pbar, flag, total;
+  __host__ __device__ MmaSmem(int stages, size_t slice_bytes) {
+    row_stride = slice_bytes + 16;
+    ring = 0;
+    w3 = ring + (size_t)stages * BLK_B * row_stride;                // w_hi, w_mid, w_lo, one zero row
+    redG = w3 + 4 * row_stride;                                     // [2][slots][64]
+    redP = redG + 2 * (size_t)MMA_SLOTS * MMA_G_VALS * sizeof(float);  // [2][slots][32]
+    totG = redP + 2 * (size_t)MMA_SLOTS * MMA_P_VALS * sizeof(float);  // [64]
+    gam = totG + 64 * sizeof(float);                                // gamma_0..7, 1 - a^nv, stop
+    tab = gam + 16 * sizeof(float);                                 // [48]
+    jet = tab + 3 * 16 * sizeof(float);                             // [8] float4
+    bars = jet + 8 * 4 * sizeof(float);                             // ring barriers [8]
+    pbar = bars + 8 * sizeof(unsigned long long);                   // partial-sum barriers [2]
+    flag = pbar + 2 * sizeof(unsigned long long);
+    total = flag + 16;
+  }
+};
+
+// 8-byte store into the shared memory of a CTA of the cluster; its 8 bytes are counted on that CTA's barrier `mbar`
+// (both addresses in the shared::cluster window of the same CTA).
+__device__ __forceinline__ void st_async_f32x2(uint32_t addr, float a, float b, uint32_t mbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr),
+               "f"(a), "f"(b), "r"(mbar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(unsigned long long* bar, uint32_t parity) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(a), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Later asynchronous-proxy writes (bulk copies) to shared memory are ordered after this thread's earlier stores.
+__device__ __forceinline__ void fence_proxy_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Two fp32 -> packed bf16 (round to nearest even); the low half holds `lo`, the high half `hi`.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+template <int LOSS>
+__global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const ClusterParams cp) {
+  constexpr int B = BLK_B;
+  extern __shared__ __align__(16) unsigned char smem[];
+  const BlockParams& bp = cp.b;
+  const ChainParams& p = bp.c;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int math_warps = (blockDim.x >> 5) - 2;
+  const int S = bp.stages;
+  const uint32_t C = cluster_nctarank(), rank = cluster_ctarank();
+  const int j = p.order[blockIdx.x / C];
+  const long long n_run = p.n_steps[j];
+  const long long d = p.d;
+  const long long chunks = d / 8;
+  const long long chunk0 = (long long)rank * cp.chunks_per_cta;
+  const long long chunk_end = chunk0 + cp.chunks_per_cta < chunks ? chunk0 + cp.chunks_per_cta : chunks;
+  const int my_chunks = (int)(chunk_end > chunk0 ? chunk_end - chunk0 : 0);
+  const size_t slice_bytes = (size_t)cp.chunks_per_cta * 16;
+  const size_t ld_bytes = (size_t)p.ld * 2;
+  const MmaSmem L(S, slice_bytes);
+  const size_t row_stride = L.row_stride;
+  unsigned char* ring = smem + L.ring;
+  unsigned char* w3 = smem + L.w3;
+  float* redG = (float*)(smem + L.redG);
+  float* redP = (float*)(smem + L.redP);
+  float* totG = (float*)(smem + L.totG);
+  float* gam = (float*)(smem + L.gam);
+  float* tab = (float*)(smem + L.tab);  // [0..8] a^k, [16..24] eta / a^{k+1}, [32..40] 1 - a^k
+  float4* jets = (float4*)(smem + L.jet);
+  unsigned long long* bars = (unsigned long long*)(smem + L.bars);
+  unsigned long long* pbar = (unsigned long long*)(smem + L.pbar);
+  volatile int* give_up = (volatile int*)(smem + L.flag);
+  const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes + (size_t)chunk0 * 16;
+  const float* yshard = p.y + p.shard_off[j];
+  const uint32_t* idx = p.idx + p.idx_off[j];
+  const long long nb = (n_run + B - 1) / B;
+
+  // ---- set-up: tables, barriers, zeroed ring / model rows / partial-sum tables ------------------------------------
+  if (threadIdx.x <= B) {  // power tables in fp64, rounded once
+    const double a = 1.0 - bp.eta_lambda;
+    double pw = 1.0;
+    for (int k = 0; k < (int)threadIdx.x; ++k) pw *= a;
+    tab[threadIdx.x] = (float)pw;
+    tab[16 + threadIdx.x] = (float)((double)p.eta0 / (pw * a));
+    tab[32 + threadIdx.x] = (float)(1.0 - pw);
+  }
+  if (threadIdx.x == 32) {
+    for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
+    mbar_init(&pbar[0], 1);
+    mbar_init(&pbar[1], 1);
+    *give_up = 0;
+    mbar_fence_init();
+  }
+  {
+    // everything from the ring up to the end of the partial-sum tables starts at zero: columns beyond a slice, the
+    // zero row of the model rows and the table slots that no math warp writes are never written later
+    uint4* z = (uint4*)smem;
+    const int n16 = (int)(L.totG / 16);
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  fence_proxy_async_shared();
+  __syncthreads();
+
+  if (warp == 0) {
+    // =========================== recurrence warp ========================================================
+    const int n = lane & (B - 1);
+    float y_nxt = 0.0f;
+    uint32_t id_nxt = 0u;
+    if (nb > 0) y_nxt = yshard[idx[n]];
+    if (nb > 1) id_nxt = idx[B + n];
+    float apw[B], cfac[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+    const uint32_t expect_bytes = C * (uint32_t)math_warps * MMA_SLOT_BYTES;
+    cluster_barrier();  // start-up: every CTA of the cluster runs and has set up its shared memory
+
+    for (long long b = 0; b < nb; ++b) {
+      const int nv = (int)((n_run - b * B) < (long long)B ? (n_run - b * B) : (long long)B);
+      const int q = (int)(b & 1);
+      if (lane == 0) mbar_arrive_expect_tx(&pbar[q], expect_bytes);
+      const float y_cur = y_nxt;
+      if (b + 1 < nb) y_nxt = yshard[id_nxt];
+      if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
+      const float a_nv = tab[nv], dl_nv = tab[32 + nv];
+      float yv[B], sc[B], cf[B];
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+        if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
+          sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
+          cf[m] = -yv[m] * cfac[m];
+        } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
+          sc[m] = yv[m] * apw[m];
+          cf[m] = -yv[m] * cfac[m];
+        } else {  // g = t - y, t = a^n (...)
+          sc[m] = apw[m];
+          cf[m] = cfac[m];
+        }
+        if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
+      }
+      // ---- wait (bounded) for the partial sums of block b from every math warp of the cluster ------------------
+      {
+        const uint32_t parity = (uint32_t)((b >> 1) & 1);
+        bool landed = false;
+        for (long long i = 0; i < bp.spin_limit; ++i) {
+          if (mbar_try_wait_cluster(&pbar[q], parity)) { landed = true; break; }
+          if (*give_up) break;
+        }
+        if (!landed && !*give_up) {
+          set_status(p.status, DEV_TIMEOUT, 2, (long long)blockIdx.x);
+          for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
+        }
+      }
+      const int stop = *give_up;
+      const float* rG = redG + (size_t)q * MMA_SLOTS * MMA_G_VALS;
+      const float* rP = redP + (size_t)q * MMA_SLOTS * MMA_P_VALS;
+      float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
+      {
+        float g0[MMA_SLOTS], g1[MMA_SLOTS];
+#pragma unroll
+        for (int w = 0; w < MMA_SLOTS; ++w) { g0[w] = rG[w * 64 + lane]; g1[w] = rG[w * 64 + 32 + lane]; }
+#pragma unroll
+        for (int h = MMA_SLOTS / 2; h >= 1; h >>= 1)
+#pragma unroll
+          for (int w = 0; w < h; ++w) { g0[w] += g0[w + h]; g1[w] += g1[w + h]; }
+        totG[lane] = g0[0];
+        totG[32 + lane] = g1[0];
+        __syncwarp();
+#pragma unroll
+        for (int n2 = 1; n2 < B; ++n2) {
+          const float4 lo = *(const float4*)&totG[n2 * 8], hi = *(const float4*)&totG[n2 * 8 + 4];
+          const float row[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+          for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] = row[m] * sc[n2];
+        }
+        __syncwarp();
+      }
+      float psum;
+      {
+        float pp[MMA_SLOTS];
+#pragma unroll
+        for (int w = 0; w < MMA_SLOTS; ++w) pp[w] = rP[w * MMA_P_VALS + lane];
+#pragma unroll
+        for (int h = MMA_SLOTS / 2; h >= 1; h >>= 1)
+#pragma unroll
+          for (int w = 0; w < h; ++w) pp[w] += pp[w + h];
+        // lanes 0..7: w_hi . x_n, 8..15: w_mid . x_n, 16..23: w_lo . x_n (24..31: zero); small terms first
+        const float mid = __shfl_down_sync(0xffffffffu, pp[0], 8), lo = __shfl_down_sync(0xffffffffu, pp[0], 16);
+        psum = (lo + mid) + pp[0];  // lanes 0..7: p_n
+      }
+      float t[B], beta[B];
+#pragma unroll
+      for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
+      if (LOSS == LOSS_LOGISTIC) {
+        // lane n < 8 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
+        if (lane < B) jets[lane] = logistic_jet(y_cur * tab[n] * 1.4426950408889634f * psum);
+        __syncwarp();
+        float4 jet[B];
+        float dlt[B];
+#pragma unroll
+        for (int m = 0; m < B; ++m) {
+          jet[m] = jets[m];
+          dlt[m] = 0.0f;
+        }
+        float dmax = 0.0f;
+#pragma unroll
+        for (int m = 0; m < B; ++m) {
+          dmax = fmaxf(dmax, fabsf(dlt[m]));
+          beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
+#pragma unroll
+          for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
+        }
+        if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
+#pragma unroll 1
+          for (int m = 0; m < B; ++m) {
+            float tm_ = 0.0f, cfm = 0.0f;
+#pragma unroll
+            for (int k = 0; k < B; ++k)
+              if (k == m) { tm_ = t[k]; cfm = cf[k]; }
+            const float bm = cfm * logistic_factor(tm_);
+#pragma unroll
+            for (int k = 0; k < B; ++k)
+              if (k == m) beta[k] = bm;
+#pragma unroll
+            for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+              for (int k = 0; k < n2; ++k)
+                if (k == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + k], t[n2]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int m = 0; m < B; ++m) {
+          if (LOSS == LOSS_HINGE) {
+            beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+          } else {
+            beta[m] = cf[m] * (t[m] - yv[m]);
+          }
+#pragma unroll
+          for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+        }
+      }
+      // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}; [8] = 1 - a^nv; [9] = leave after this block
+      float mine = dl_nv;
+#pragma unroll
+      for (int m = 0; m < B; ++m)
+        if (lane == m) mine = beta[m] * a_nv;
+      if (lane == B + 1) mine = stop ? 1.0f : 0.0f;
+      if (lane <= B + 1) gam[lane] = mine;
+      __syncthreads();  // gamma and the decision published
+      if (stop) break;
+    }
+    cluster_barrier();  // nobody exits while a peer may still store into its shared memory
+    return;
+  }
+
+  if (warp == 1) {
+    // =========================== copy warp ==============================================================
+    // Lane m < 8 requests this CTA's column slice of row m of a block as one bulk copy; the eight copies complete on
+    // the stage's barrier. A stage is refilled after the CTA barrier of the following block: by then every math
+    // warp of this CTA has applied the update that was the last read of the stage.
+    const uint32_t copy_bytes = (uint32_t)my_chunks * 16u;
+    uint32_t id_next = 0u;
+    auto peek = [&](long long blk) {
+      if (lane < B && blk < nb) id_next = idx[blk * B + lane];
+    };
+    auto request = [&](long long blk, int stg) {
+      if (blk < nb && blk != bp.drop_block && copy_bytes > 0) {
+        if (lane == 0) mbar_arrive_expect_tx(&bars[stg], B * copy_bytes);
+        __syncwarp();
+        if (lane < B)
+          bulk_copy_g2s(ring + ((size_t)stg * B + lane) * row_stride, shard + (size_t)id_next * ld_bytes, copy_bytes, &bars[stg]);
+      }
+    };
+    long long requested = 0;
+    for (int s = 0; s < S; ++s) {
+      peek(s);
+      request(s, s);
+      ++requested;
+    }
+    peek(requested);
+    cluster_barrier();  // start-up
+    int st = 0;         // stage of block b - 1
+    long long b = 0;
+    bool stop = false;
+    for (; b < nb; ++b) {
+      __syncthreads();
+      if (gam[B + 1] != 0.0f) { stop = true; break; }
+      if (b >= 1) {
+        request(requested, st);
+        ++requested;
+        peek(requested);
+        st = (st + 1 == S) ? 0 : st + 1;
+      }
+    }
+    if (stop && copy_bytes > 0) {
+      // leave no copy in flight into this CTA's shared memory: wait (bounded) on the stage of every block that was
+      // requested and may not have landed yet
+      long long blk = b - 1 > 0 ? b - 1 : 0;
+      for (; blk < requested && blk < nb; ++blk)
+        if (blk != bp.drop_block) mbar_wait_bounded(&bars[blk % S], (uint32_t)((blk / S) & 1), bp.spin_limit);
+    }
+    cluster_barrier();
+    return;
+  }
+
+  // ============================= math warps ==============================================================
+  const int mw = warp - 2;
+  const int lc = mw * 32 + lane;  // this thread's chunk within the CTA's slice
+  const bool act = lc < my_chunks;
+  const int warp_chunks = my_chunks - mw * 32 < 0 ? 0 : (my_chunks - mw * 32 > 32 ? 32 : my_chunks - mw * 32);
+  const int ksteps = (warp_chunks + 1) >> 1;  // 16 columns (two chunks) per tensor-core instruction
+  float2 w2[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) w2[i] = make_float2(0.0f, 0.0f);
+  if (act) {
+    const long long c0 = (chunk0 + lc) * 8;
+    const float* src = p.resume ? (p.W + (size_t)j * d + c0) : (p.w0 ? p.w0 + c0 : nullptr);
+    if (src) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w2[i] = make_float2(src[2 * i], src[2 * i + 1]);
+    }
+  }
+  // the thread's 8 model values as three bf16 rows: w = hi + mid + lo (each remainder is exact in fp32)
+  auto publish_model = [&]() {
+    if (act) {
+      uint32_t hi[4], mid[4], lo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        hi[i] = pack_bf16x2(w2[i].x, w2[i].y);
+        const float rx = w2[i].x - __uint_as_float(hi[i] << 16), ry = w2[i].y - __uint_as_float(hi[i] & 0xffff0000u);
+        mid[i] = pack_bf16x2(rx, ry);
+        const float sx = rx - __uint_as_float(mid[i] << 16), sy = ry - __uint_as_float(mid[i] & 0xffff0000u);
+        lo[i] = pack_bf16x2(sx, sy);
+      }
+      *(uint4*)(w3 + 0 * row_stride + (size_t)lc * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *(uint4*)(w3 + 1 * row_stride + (size_t)lc * 16) = make_uint4(mid[0], mid[1], mid[2], mid[3]);
+      *(uint4*)(w3 + 2 * row_stride + (size_t)lc * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    __syncwarp();
+  };
+  publish_model();
+  // tile addresses of the tensor-core operand loads: lanes 8i..8i+7 give the 8 row addresses of tile i; tiles 0 and 2
+  // are the staged rows (columns +0 and +8), tiles 1 and 3 the model rows (hi, mid, lo, then the zero row)
+  const int tile = lane >> 3, trow = lane & 7;
+  const size_t tile_col_bytes = (size_t)mw * 512 + (size_t)(tile >> 1) * 16;
+  const size_t x_off = (size_t)trow * row_stride + tile_col_bytes;
+  const unsigned char* w_src = w3 + (size_t)(trow < 3 ? trow : 3) * row_stride + tile_col_bytes;
+  const int slot = (int)rank * math_warps + mw;
+  cluster_barrier();  // start-up
+
+  int st = 0;
+  uint32_t par = 0u;
+  for (long long b = 0; b < nb; ++b) {
+    if (my_chunks > 0 && !mbar_wait_bounded(&bars[st], par, bp.spin_limit)) {
+      set_status(p.status, DEV_TIMEOUT, 1, (long long)blockIdx.x);
+      for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
+    }
+    const unsigned char* stage = ring + (size_t)st * B * row_stride;
+    // ---- [G_b ; p_b parts] over this warp's columns ------------------------------------------------------------
+    float ca[4] = {0.0f, 0.0f, 0.0f, 0.0f}, cb[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    {
+      const unsigned char* src = (tile & 1) ? w_src : stage + x_off;
+#pragma unroll 4
+      for (int ks = 0; ks < ksteps; ks += 2) {
+        uint32_t q0[4], q1[4];
+        ldmatrix_x4(q0, src + (size_t)ks * 32);
+        mma_bf16_m16n8k16(ca, q0[0], q0[1], q0[2], q0[3], q0[0], q0[2]);
+        if (ks + 1 < ksteps) {
+          ldmatrix_x4(q1, src + (size_t)(ks + 1) * 32);
+          mma_bf16_m16n8k16(cb, q1[0], q1[1], q1[2], q1[3], q1[0], q1[2]);
+        }
+      }
+    }
+    const float c0 = ca[0] + cb[0], c1 = ca[1] + cb[1], c2 = ca[2] + cb[2], c3 = ca[3] + cb[3];
+    {
+      // accumulator rows 0..7: lane l holds G[l / 4][2 (l % 4) .. +1]; rows 8..10 (lanes 0..11): the parts of p
+      const int q = (int)(b & 1);
+      float* dg = redG + ((size_t)q * MMA_SLOTS + slot) * MMA_G_VALS + lane * 2;
+      float* dp = redP + ((size_t)q * MMA_SLOTS + slot) * MMA_P_VALS + lane * 2;
+      for (uint32_t rr = 0; rr < C; ++rr) {
+        const uint32_t bar = map_shared_rank(&pbar[q], rr);
+        st_async_f32x2(map_shared_rank(dg, rr), c0, c1, bar);
+        if (lane < 12) st_async_f32x2(map_shared_rank(dp, rr), c2, c3, bar);
+      }
+    }
+    __syncthreads();  // gamma_b and the decision are in gam
+    if (gam[B + 1] != 0.0f) break;
+    // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m, then the model rows again -----------------------------------------
+    if (act) {
+      float2 ngm2[B];
+#pragma unroll
+      for (int m = 0; m < B; ++m) {
+        const float g = -gam[m];
+        ngm2[m] = make_float2(g, g);
+      }
+      const float ndl = -gam[B];
+      const float2 ndl2 = make_float2(ndl, ndl);
+      uint4 raw[B];
+#pragma unroll
+      for (int m = 0; m < B; ++m) raw[m] = *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float2 wv = __ffma2_rn(ndl2, w2[i], w2[i]);
+#pragma unroll
+        for (int m = 0; m < B; ++m) wv = __ffma2_rn(ngm2[m], XPairs<__nv_bfloat16>::get(raw[m], i), wv);
+        w2[i] = wv;
+      }
+    }
+    publish_model();
+    if (++st == S) { st = 0; par ^= 1u; }
+  }
+  cluster_barrier();
+
+  if (act) {
+    const long long c0 = (chunk0 + lc) * 8;
+    float* dst = p.W + (size_t)j * d + c0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      dst[2 * i] = w2[i].x;
+      dst[2 * i + 1] = w2[i].y;
+    }
+  }
+}
+
+}  // namespace wpsgd

@@ -11,7 +11,9 @@
 #include <vector>
 
 #include "chain_block.cuh"
+#include "chain_cluster.cuh"
 #include "chain_csr.cuh"
+#include "chain_mma.cuh"
 #include "chain_tc.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
@@ -65,6 +67,7 @@ struct wpsgd_ctx {
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
   int opt_tc_gram = 0;
+  int opt_chunks_per_thread = 0;  // cluster kernel: 16-byte chunks of a row per math thread (0: chosen here)
   int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
   int opt_timing = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -414,6 +417,171 @@ wpsgd_status launch_tc(wpsgd_ctx* c, const ChainParams& p, int R, int stages) {
   return R == 1 ? launch_tc_r<1>(c, bp, smem) : launch_tc_r<2>(c, bp, smem);
 }
 
+// ---- blocked kernel with the columns of a chain split over a thread-block cluster -------------------------------
+struct ClusterShape {
+  int C = 1, cpc = 0, R = 1, math_warps = 1, stages = 2, min_blocks = 1;
+};
+
+// Shape of the cluster launch: C CTAs per chain (a power of two up to 8, the portable cluster size), cpc chunks of
+// a row per CTA, R chunks per math thread. Aim: about two CTAs per SM over the whole grid, so that the SMs of
+// finished chains keep working for the long ones, and at least one full warp of chunks per CTA.
+template <typename XT>
+bool cluster_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
+  constexpr int V = XVec<XT>::V;
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / V;
+  if (chunks < 1) return false;
+  int C = c->opt_cluster;
+  if (C <= 0) {
+    C = 1;
+    while (C < 8 && (long long)c->k * (C * 2) <= 2 * 148 && chunks / (C * 2) >= 32) C *= 2;
+  }
+  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
+  const long long cpc = (chunks + C - 1) / C;
+  if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
+  int R = c->opt_chunks_per_thread;
+  if (R <= 0) R = cpc > 64 ? 2 : 1;
+  if (R != 1 && R != 2) return false;
+  const long long mw = (cpc + 32 * R - 1) / (32 * R);
+  if (mw > 8 || mw * C > CL_MAX_SLOTS) return false;
+  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
+  // two CTAs per SM when the ring allows it
+  const size_t per_cta_two = (size_t)(227 * 1024) / 2 - 1024;
+  int s2 = stages;
+  while (s2 >= 3 && ClusterSmem(s2, (size_t)cpc * 16).total > per_cta_two) --s2;
+  int min_blocks = 1;
+  if (s2 >= 3 && ClusterSmem(s2, (size_t)cpc * 16).total <= per_cta_two) {
+    stages = s2;
+    min_blocks = 2;
+  } else {
+    while (stages >= 2 && ClusterSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
+    if (stages < 2) return false;
+  }
+  out->C = C;
+  out->cpc = (int)cpc;
+  out->R = R;
+  out->math_warps = (int)mw;
+  out->stages = stages;
+  out->min_blocks = min_blocks;
+  return true;
+}
+
+template <typename XT, int R, int MAXMW, int MINB>
+wpsgd_status launch_cluster_r(wpsgd_ctx* c, const ClusterParams& cp, const ClusterShape& sh, size_t smem) {
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
+    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)sh.C;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_cluster_kernel<XT, R, LOSS_HINGE, MAXMW, MINB>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_cluster_kernel<XT, R, LOSS_LOGISTIC, MAXMW, MINB>);
+    default: return go(chain_cluster_kernel<XT, R, LOSS_SQUARED, MAXMW, MINB>);
+  }
+}
+
+template <typename XT>
+wpsgd_status launch_cluster(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
+  ClusterParams cp;
+  cp.b.c = p;
+  cp.b.stages = sh.stages;
+  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  cp.b.spin_limit = c->opt_spin_limit;
+  cp.b.drop_block = c->opt_drop_block;
+  cp.b.group_order = nullptr;
+  cp.chunks_per_cta = sh.cpc;
+  const size_t smem = ClusterSmem(sh.stages, (size_t)sh.cpc * 16).total;
+  if (sh.R == 1) return launch_cluster_r<XT, 1, 8, 1>(c, cp, sh, smem);
+  if (sh.math_warps <= 4 && sh.min_blocks >= 2) return launch_cluster_r<XT, 2, 4, 2>(c, cp, sh, smem);
+  return launch_cluster_r<XT, 2, 8, 1>(c, cp, sh, smem);
+}
+
+// ---- bf16 rows: Gram block and margins on the tensor cores, columns split over a cluster -------------------------------
+bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / 8;
+  if (chunks < 1) return false;
+  int C = c->opt_cluster;
+  if (C <= 0) {
+    // about two CTAs per SM over the whole grid, at least two full warps of chunks per CTA
+    C = 1;
+    while (C < 8 && (long long)c->k * (C * 2) <= 2 * 148 && chunks / (C * 2) >= 64) C *= 2;
+    while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;  // a CTA takes at most 8 math warps of 32 chunks
+  }
+  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
+  const long long cpc = (chunks + C - 1) / C;
+  if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
+  const long long mw = (cpc + 31) / 32;
+  if (mw > 8 || mw * C > MMA_SLOTS) return false;
+  // ring depth: as deep as asked for (default 4) while two CTAs still share an SM; else one CTA per SM
+  const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
+  int want = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
+  int stages = want;
+  while (stages > 2 && MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) --stages;
+  if (MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) {
+    stages = want;
+    while (stages >= 2 && MmaSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
+    if (stages < 2) return false;
+  }
+  out->C = C;
+  out->cpc = (int)cpc;
+  out->R = 1;
+  out->math_warps = (int)mw;
+  out->stages = stages;
+  out->min_blocks = 2;
+  return true;
+}
+
+wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
+  ClusterParams cp;
+  cp.b.c = p;
+  cp.b.stages = sh.stages;
+  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  cp.b.spin_limit = c->opt_spin_limit;
+  cp.b.drop_block = c->opt_drop_block;
+  cp.b.group_order = nullptr;
+  cp.chunks_per_cta = sh.cpc;
+  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16).total;
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
+    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)sh.C;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_mma_kernel<LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_mma_kernel<LOSS_LOGISTIC>);
+    default: return go(chain_mma_kernel<LOSS_SQUARED>);
+  }
+}
+
 // blocked kernel, one warp per node (small d)
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
@@ -510,6 +678,22 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
+  }
+  if (variant == 8) {
+    ClusterShape sh;
+    if (sizeof(XT) != 2 || !mma_kernel_fits(c, aligned, &sh))
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "tensor-core cluster kernel needs bf16 rows, 16-byte aligned, a constant step size, eta*lambda <= 0.25, a "
+                  "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
+    return launch_mma(c, p, sh);
+  }
+  if (variant == 7) {
+    ClusterShape sh;
+    if (!cluster_kernel_fits<XT>(c, aligned, &sh))
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "cluster kernel needs 16-byte aligned rows, a constant step size, eta*lambda <= 0.25, a cluster of 1, 2, 4 "
+                  "or 8 CTAs with at most 512 chunks of a row each and at most 16 math warps in all");
+    return launch_cluster<XT>(c, p, sh);
   }
   if (variant == 6 || (variant == 4 && c->opt_tc_gram == 2)) {
     int tR = 0, tstages = 0;
@@ -708,7 +892,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 6) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..6");
+    if (value < 0 || value > 8) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..8");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");
@@ -722,6 +906,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "cluster") {
     if (value < 0 || value > 16) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0..16");
     c->opt_cluster = (int)value;
+  } else if (n == "chunks_per_thread") {
+    if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "chunks_per_thread must be 0, 1 or 2");
+    c->opt_chunks_per_thread = (int)value;
   } else if (n == "sparse_threads") {
     if (value != 32) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_threads must be 32");
     c->opt_sparse_threads = (int)value;
