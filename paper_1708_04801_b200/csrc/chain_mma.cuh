@@ -305,8 +305,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
   if (warp == 1) {
     // =========================== copy warp ==============================================================
     // Lane m < 8 requests this CTA's column slice of row m of a block as one bulk copy; the eight copies complete on
-    // the stage's barrier. A stage is refilled after the CTA barrier of the following block: by then every math
-    // warp of this CTA has applied the update that was the last read of the stage.
+    // the stage's barrier. A stage is refilled right after the CTA barrier of its block: by then every math warp of
+    // this CTA has run the tensor-core pass over it and holds its own columns of the rows in registers.
     const uint32_t copy_bytes = (uint32_t)my_chunks * 16u;
     uint32_t id_next = 0u;
     auto peek = [&](long long blk) {
@@ -328,23 +328,21 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
     }
     peek(requested);
     cluster_barrier();  // start-up
-    int st = 0;         // stage of block b - 1
+    int st = 0;         // stage of block b
     long long b = 0;
     bool stop = false;
     for (; b < nb; ++b) {
       __syncthreads();
       if (gam[B + 1] != 0.0f) { stop = true; break; }
-      if (b >= 1) {
-        request(requested, st);
-        ++requested;
-        peek(requested);
-        st = (st + 1 == S) ? 0 : st + 1;
-      }
+      request(requested, st);
+      ++requested;
+      peek(requested);
+      st = (st + 1 == S) ? 0 : st + 1;
     }
     if (stop && copy_bytes > 0) {
       // leave no copy in flight into this CTA's shared memory: wait (bounded) on the stage of every block that was
       // requested and may not have landed yet
-      long long blk = b - 1 > 0 ? b - 1 : 0;
+      long long blk = b;
       for (; blk < requested && blk < nb; ++blk)
         if (blk != bp.drop_block) mbar_wait_bounded(&bars[blk % S], (uint32_t)((blk / S) & 1), bp.spin_limit);
     }
@@ -395,6 +393,11 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
   const size_t x_off = (size_t)trow * row_stride + tile_col_bytes;
   const unsigned char* w_src = w3 + (size_t)(trow < 3 ? trow : 3) * row_stride + tile_col_bytes;
   const int slot = (int)rank * math_warps + mw;
+  // shared-memory window of every CTA of the cluster (the same offsets apply inside each window)
+  const uint32_t own_base = (uint32_t)__cvta_generic_to_shared(smem);
+  uint32_t peer_base[8];
+#pragma unroll
+  for (int rr = 0; rr < 8; ++rr) peer_base[rr] = map_shared_rank(smem, (uint32_t)rr < C ? (uint32_t)rr : rank);
   cluster_barrier();  // start-up
 
   int st = 0;
@@ -406,33 +409,51 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
     }
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
     // ---- [G_b ; p_b parts] over this warp's columns ------------------------------------------------------------
-    float ca[4] = {0.0f, 0.0f, 0.0f, 0.0f}, cb[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    // eight independent accumulators (the instruction's latency is long), two rounds of eight 16-column steps
+    float acc[8][4];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[a][e] = 0.0f;
     {
       const unsigned char* src = (tile & 1) ? w_src : stage + x_off;
-#pragma unroll 4
-      for (int ks = 0; ks < ksteps; ks += 2) {
-        uint32_t q0[4], q1[4];
-        ldmatrix_x4(q0, src + (size_t)ks * 32);
-        mma_bf16_m16n8k16(ca, q0[0], q0[1], q0[2], q0[3], q0[0], q0[2]);
-        if (ks + 1 < ksteps) {
-          ldmatrix_x4(q1, src + (size_t)(ks + 1) * 32);
-          mma_bf16_m16n8k16(cb, q1[0], q1[1], q1[2], q1[3], q1[0], q1[2]);
-        }
+#pragma unroll
+      for (int round = 0; round < 2; ++round) {
+        uint32_t q[8][4];
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+          if (round * 8 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 8 + a) * 32);
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+          if (round * 8 + a < ksteps) mma_bf16_m16n8k16(acc[a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
       }
     }
-    const float c0 = ca[0] + cb[0], c1 = ca[1] + cb[1], c2 = ca[2] + cb[2], c3 = ca[3] + cb[3];
+#pragma unroll
+    for (int h = 4; h >= 1; h >>= 1)
+#pragma unroll
+      for (int a = 0; a < h; ++a)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[a][e] += acc[a + h][e];
     {
       // accumulator rows 0..7: lane l holds G[l / 4][2 (l % 4) .. +1]; rows 8..10 (lanes 0..11): the parts of p
       const int q = (int)(b & 1);
-      float* dg = redG + ((size_t)q * MMA_SLOTS + slot) * MMA_G_VALS + lane * 2;
-      float* dp = redP + ((size_t)q * MMA_SLOTS + slot) * MMA_P_VALS + lane * 2;
-      for (uint32_t rr = 0; rr < C; ++rr) {
-        const uint32_t bar = map_shared_rank(&pbar[q], rr);
-        st_async_f32x2(map_shared_rank(dg, rr), c0, c1, bar);
-        if (lane < 12) st_async_f32x2(map_shared_rank(dp, rr), c2, c3, bar);
+      const uint32_t og = (uint32_t)__cvta_generic_to_shared(redG + ((size_t)q * MMA_SLOTS + slot) * MMA_G_VALS + lane * 2) - own_base;
+      const uint32_t op = (uint32_t)__cvta_generic_to_shared(redP + ((size_t)q * MMA_SLOTS + slot) * MMA_P_VALS + lane * 2) - own_base;
+      const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&pbar[q]) - own_base;
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr) {
+        if ((uint32_t)rr < C) {
+          st_async_f32x2(peer_base[rr] + og, acc[0][0], acc[0][1], peer_base[rr] + ob);
+          if (lane < 12) st_async_f32x2(peer_base[rr] + op, acc[0][2], acc[0][3], peer_base[rr] + ob);
+        }
       }
     }
-    __syncthreads();  // gamma_b and the decision are in gam
+    // this thread's columns of the 8 rows, for the update: afterwards the stage can be refilled
+    uint4 raw[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m)
+      raw[m] = act ? *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16) : make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();  // gamma_b and the decision are in gam; every math warp is done with the stage
     if (gam[B + 1] != 0.0f) break;
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m, then the model rows again -----------------------------------------
     if (act) {
@@ -444,9 +465,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
       }
       const float ndl = -gam[B];
       const float2 ndl2 = make_float2(ndl, ndl);
-      uint4 raw[B];
-#pragma unroll
-      for (int m = 0; m < B; ++m) raw[m] = *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float2 wv = __ffma2_rn(ndl2, w2[i], w2[i]);

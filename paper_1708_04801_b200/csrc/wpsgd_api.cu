@@ -13,6 +13,7 @@
 #include "chain_block.cuh"
 #include "chain_cluster.cuh"
 #include "chain_csr.cuh"
+#include "chain_lag.cuh"
 #include "chain_mma.cuh"
 #include "chain_tc.cuh"
 #include "chain_dense.cuh"
@@ -582,6 +583,80 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   }
 }
 
+// ---- bf16 rows: lagged blocked form (margins one block behind the model), columns split over a cluster -----------------------
+bool lag_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / 8;
+  if (chunks < 1) return false;
+  int C = c->opt_cluster;
+  if (C <= 0) {
+    // a chain's speed is set by the tensor-core pass of its CTAs, so wide rows are split four ways; at least two full
+    // warps of chunks per CTA
+    C = 1;
+    while (C < 4 && chunks / (C * 2) >= 64) C *= 2;
+    while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;  // a CTA takes at most 8 math warps of 32 chunks
+  }
+  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
+  const long long cpc = (chunks + C - 1) / C;
+  if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
+  const long long mw = (cpc + 31) / 32;
+  if (mw > 8 || mw * C > LAG_SLOTS) return false;
+  // ring depth (at least 3: the blocks i, i + 1 and i + 2 are in use at the same time): as deep as asked for
+  // (default 4) while two CTAs still share an SM; else one CTA per SM
+  const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
+  int want = c->opt_stages > 0 ? std::min(std::max(c->opt_stages, 3), 8) : 4;
+  int stages = want;
+  while (stages > 3 && LagSmem(stages, (size_t)cpc * 16).total > two_per_sm) --stages;
+  if (LagSmem(stages, (size_t)cpc * 16).total > two_per_sm) {
+    stages = want;
+    while (stages >= 3 && LagSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
+    if (stages < 3) return false;
+  }
+  out->C = C;
+  out->cpc = (int)cpc;
+  out->R = 1;
+  out->math_warps = (int)mw;
+  out->stages = stages;
+  out->min_blocks = 1;
+  return true;
+}
+
+wpsgd_status launch_lag(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
+  ClusterParams cp;
+  cp.b.c = p;
+  cp.b.stages = sh.stages;
+  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  cp.b.spin_limit = c->opt_spin_limit;
+  cp.b.drop_block = c->opt_drop_block;
+  cp.b.group_order = nullptr;
+  cp.chunks_per_cta = sh.cpc;
+  const size_t smem = LagSmem(sh.stages, (size_t)sh.cpc * 16).total;
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
+    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)sh.C;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_lag_kernel<LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_lag_kernel<LOSS_LOGISTIC>);
+    default: return go(chain_lag_kernel<LOSS_SQUARED>);
+  }
+}
+
 // blocked kernel, one warp per node (small d)
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
@@ -678,6 +753,14 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
+  }
+  if (variant == 9) {
+    ClusterShape sh;
+    if (sizeof(XT) != 2 || !lag_kernel_fits(c, aligned, &sh))
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "lagged cluster kernel needs bf16 rows, 16-byte aligned, a constant step size, eta*lambda <= 0.25, a "
+                  "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
+    return launch_lag(c, p, sh);
   }
   if (variant == 8) {
     ClusterShape sh;
@@ -892,7 +975,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 8) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..8");
+    if (value < 0 || value > 9) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..9");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");

@@ -318,10 +318,14 @@ def test_cluster_kernel_bounded_wait_reports_timeout_and_context_survives(P, d, 
     assert rel_l2(v, ov) <= 1e-4
 
 
-# ---- tensor-core cluster kernel (bf16 rows): Gram block and margins from mma, model split into three bf16 rows ------------
+# ---- tensor-core cluster kernels (bf16 rows). 8: Gram block and margins from mma, model split into three bf16 rows;
+# 9: lagged form (margins one block behind the model), Gram block and cross-block products from mma ---------------------
+TC_VARIANTS = [8, 9]
+
 @pytest.mark.parametrize("cluster", [1, 2, 4])
 @pytest.mark.parametrize("d", [480, 488, 8, 264])
-def test_mma_kernel_ragged_shapes(P, cluster, d):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_ragged_shapes(P, cluster, d, variant):
     # 60 / 61 / 1 / 33 chunks of 8 columns: odd chunk counts leave half a 16-column tile empty, the last CTA of a
     # cluster owns a ragged slice, and with d = 8 only one CTA can exist
     if d == 8 and cluster > 1:
@@ -330,44 +334,48 @@ def test_mma_kernel_ragged_shapes(P, cluster, d):
     wl.n_steps[2] = 0
     wl.w0 = torch.full((d,), 0.05)
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": 8, "cluster": cluster})
+    assert_parity(P, wl, {"dense_variant": variant, "cluster": cluster})
 
 
 @pytest.mark.parametrize("d,cluster", [(4096, 2), (4096, 4), (2048, 1), (4096, 8), (3008, 2), (1024, 8)])
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
-def test_mma_kernel_losses_and_widths(P, d, cluster, loss):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_losses_and_widths(P, d, cluster, loss, variant):
     wl = wi.config2(k=3, d=d, m=48, base_steps=210)
     wl.loss = loss
     if loss == SQUARED:
         wl.y = (wl.y * 0.3).contiguous()
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": 8, "cluster": cluster})
+    assert_parity(P, wl, {"dense_variant": variant, "cluster": cluster})
 
 
 @pytest.mark.parametrize("n_steps", [(1, 7, 8), (9, 15, 16), (17, 0, 64), (333, 250, 3)])
 @pytest.mark.parametrize("stages", [2, 3, 4])
-def test_mma_kernel_block_boundaries_and_ring_depths(P, n_steps, stages):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_block_boundaries_and_ring_depths(P, n_steps, stages, variant):
     wl = wi.config2(k=3, d=1024, m=64, base_steps=8)
     wl.n_steps = np.array(n_steps, dtype=np.int64)
     wl.w0 = torch.full((1024,), 0.1)
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": 8, "cluster": 2, "stages": stages})
+    assert_parity(P, wl, {"dense_variant": variant, "cluster": 2, "stages": stages})
 
 
-def test_mma_kernel_model_split_keeps_fp32_accuracy(P):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_model_split_keeps_fp32_accuracy(P, variant):
     # a model with a wide spread of magnitudes (w0 from 1e-6 to 1e3): the three bf16 rows must carry all 24 bits of
     # every entry, or the margins of the first steps are off by far more than the tolerance
     wl = wi.config3(k=4, d=2048, m=64, n_lo=40, n_hi=90)
     g = torch.Generator().manual_seed(11)
     wl.w0 = (torch.randn(2048, generator=g) * torch.logspace(-6, 3, 2048)).contiguous()
-    assert_parity(P, wl, {"dense_variant": 8, "cluster": 2})
+    assert_parity(P, wl, {"dense_variant": variant, "cluster": 2})
 
 
-def test_mma_kernel_default_shape_and_continue(P):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_default_shape_and_continue(P, variant):
     wl_cpu = wi.small(3)
     wl = wl_cpu.to("cuda")
     with P.Context(wl.k, wl.d) as ctx:
-        ctx.set_option("dense_variant", 8)
+        ctx.set_option("dense_variant", variant)
         first = np.minimum(wl.n_steps, 301)
         ctx.run(wl.X, wl.y, wl.shard_off, first, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
         ctx.continue_(wl.X, wl.y, wl.shard_off, wl.n_steps - first)
@@ -378,26 +386,28 @@ def test_mma_kernel_default_shape_and_continue(P):
         assert rel_l2(seg[j], oW[j]) <= 1e-4
 
 
-def test_mma_kernel_limits(P):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_limits(P, variant):
     wl = wi.config2(k=2, d=64, m=16, base_steps=20)  # fp32 rows
     with pytest.raises(P.WpsgdError) as e:
-        gpu_solve(P, wl, {"dense_variant": 8})
+        gpu_solve(P, wl, {"dense_variant": variant})
     assert e.value.status_name == "UNSUPPORTED"
     wl.X = wl.X.to(torch.bfloat16)  # 8 chunks: a cluster of 8 needs 8 non-empty slices; 16 CTAs cannot exist
     with pytest.raises(P.WpsgdError) as e:
-        gpu_solve(P, wl, {"dense_variant": 8, "cluster": 16})
+        gpu_solve(P, wl, {"dense_variant": variant, "cluster": 16})
     assert e.value.status_name == "UNSUPPORTED"
 
 
 @pytest.mark.parametrize("d,cluster", [(1024, 1), (4096, 2), (4096, 4)])
-def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, cluster):
+@pytest.mark.parametrize("variant", TC_VARIANTS)
+def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, cluster, variant):
     # Failure detection without a fault: the rows of block 3 are never requested (test hook), so the bounded wait
     # for them runs out; every CTA of the cluster is told, all leave in step, and the next run is clean.
     wl_cpu = wi.config2(k=3, d=d, m=32, base_steps=120)
     wl_cpu.X = wl_cpu.X.to(torch.bfloat16)
     wl = wl_cpu.to("cuda")
     with P.Context(wl.k, wl.d) as ctx:
-        ctx.set_option("dense_variant", 8)
+        ctx.set_option("dense_variant", variant)
         ctx.set_option("cluster", cluster)
         ctx.set_option("spin_limit", 2000)
         ctx.set_option("test_drop_block", 3)
@@ -415,7 +425,7 @@ def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, clus
 
 
 # ---- logistic loss: blocks whose steps move the margins far take the direct evaluation ---------------------------------
-@pytest.mark.parametrize("variant,d", [(4, 1024), (5, 128), (7, 1024), (8, 1024)])
+@pytest.mark.parametrize("variant,d", [(4, 1024), (5, 128), (7, 1024), (8, 1024), (9, 1024)])
 def test_logistic_large_steps_between_correlated_rows(P, variant, d):
     # rows that are nearly parallel (large Gram entries) and a large step size: inside a block of 8 samples the
     # margins move by much more than the range of the cubic expansion of the logistic factor
@@ -424,7 +434,7 @@ def test_logistic_large_steps_between_correlated_rows(P, variant, d):
     base = torch.randn(d, generator=g) / np.sqrt(d)
     wl.X = (2.0 * base[None, :] + 0.3 * wl.X).contiguous()
     wl.eta0 = 0.4
-    if variant == 8:
+    if variant >= 8:
         wl.X = wl.X.to(torch.bfloat16)
     assert_parity(P, wl, {"dense_variant": variant})
 
