@@ -29,9 +29,13 @@
 // count holds for q (sent for block i + 2 after gamma_i; every recurrence warp is at block i - 1 or later). gamma
 // itself stays inside its CTA and is double buffered: gamma_{i+2} needs q_{i+2}, which is formed after gamma_i was read.
 //
-// Every wait is bounded and also leaves when the give-up flag is set. A wait that runs out sets the status word and
-// the flag of every CTA of the cluster; each warp then leaves its loop on its own and all threads meet at one final
-// cluster barrier, so no CTA exits while a peer may still store into its shared memory.
+// gamma_b goes from the recurrence warp to the math warps of its CTA through a named hardware barrier (the math
+// warps park there without polling; the recurrence warp only arrives). Every wait on data from elsewhere (rows,
+// partial sums, free stages) is a bounded poll that also ends when the give-up flag is set. A wait that
+// runs out sets the status word and the flag of every CTA of the cluster; math warps carry on with whatever is in
+// shared memory until the recurrence warp, which samples the flag once per block, publishes "stop" with gamma: it
+// never leaves without arriving at the barrier, so nobody is left parked. All threads meet at one final cluster
+// barrier, so no CTA exits while a peer may still store into its shared memory.
 #pragma once
 
 #include "chain_mma.cuh"
@@ -45,26 +49,33 @@ constexpr uint32_t LAG_GC_BYTES = LAG_GC_VALS * sizeof(float);  // one math warp
 constexpr uint32_t LAG_Q_BYTES = BLK_B * sizeof(float);
 
 struct LagSmem {
-  size_t row_stride, ring, redGC, redQ, tot, gam, tab, jet, full, fre, gbar, qbar, gambar, flag, total;
+  size_t row_stride, ring, redGC, redQ, tot, gam, tab, jet, full, fre, gbar, qbar, flag, total;
   __host__ __device__ LagSmem(int stages, size_t slice_bytes) {
     row_stride = slice_bytes + 16;
     ring = 0;
     redGC = ring + (size_t)stages * BLK_B * row_stride;                   // [4][slots][128]
     redQ = redGC + LAG_DEPTH * (size_t)LAG_SLOTS * LAG_GC_VALS * sizeof(float);   // [4][slots][8]
     tot = redQ + LAG_DEPTH * (size_t)LAG_SLOTS * BLK_B * sizeof(float);   // [128]
-    gam = tot + LAG_GC_VALS * sizeof(float);                              // [2][16]: gamma_0..7, 1 - a^nv
+    gam = tot + LAG_GC_VALS * sizeof(float);                              // [2][16]: gamma_0..7, 1 - a^nv, stop
     tab = gam + 2 * 16 * sizeof(float);                                   // [48]
     jet = tab + 3 * 16 * sizeof(float);                                   // [8] float4
     full = jet + 8 * 4 * sizeof(float);                                   // [8] rows of a stage have landed
     fre = full + 8 * sizeof(unsigned long long);                          // [8] stage may be refilled
     gbar = fre + 8 * sizeof(unsigned long long);                          // [4] G / C partial sums
     qbar = gbar + LAG_DEPTH * sizeof(unsigned long long);                 // [4] q partial sums
-    gambar = qbar + LAG_DEPTH * sizeof(unsigned long long);               // [2] gamma published
-    flag = gambar + 2 * sizeof(unsigned long long);
+    flag = qbar + LAG_DEPTH * sizeof(unsigned long long);
     total = flag + 16;
   }
 };
 
+// Named hardware barrier `id` of the CTA for `nthreads` threads: sync parks the warp until all have arrived, arrive
+// only reports. Stores before an arrive are visible after the matching sync.
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int nthreads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
   const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a) : "memory");
@@ -74,11 +85,29 @@ __device__ __forceinline__ void st_async_f32(uint32_t addr, float a, uint32_t mb
                "r"(mbar)
                : "memory");
 }
+// Non-blocking look at a barrier phase (try_wait may hold the thread for a while even when the phase is complete).
+__device__ __forceinline__ bool mbar_test_wait(unsigned long long* bar, uint32_t parity, bool cluster_scope) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+  uint32_t ok;
+  if (cluster_scope)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity)
+        : "memory");
+  return ok != 0;
+}
 // Bounded wait that also ends when the give-up flag is set; true when the phase completed.
 __device__ __forceinline__ bool mbar_wait_or_give_up(unsigned long long* bar, uint32_t parity, long long limit,
                                                      volatile int* give_up, bool cluster_scope) {
   for (long long i = 0; i < limit; ++i) {
-    if (cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    if (mbar_test_wait(bar, parity, cluster_scope)) return true;
     if (*give_up) return false;
   }
   return false;
@@ -116,7 +145,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
   unsigned long long* fre = (unsigned long long*)(smem + L.fre);
   unsigned long long* gbar = (unsigned long long*)(smem + L.gbar);
   unsigned long long* qbar = (unsigned long long*)(smem + L.qbar);
-  unsigned long long* gambar = (unsigned long long*)(smem + L.gambar);
   volatile int* give_up = (volatile int*)(smem + L.flag);
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes + (size_t)chunk0 * 16;
   const float* yshard = p.y + p.shard_off[j];
@@ -141,8 +169,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
       mbar_init(&gbar[q], 1);
       mbar_init(&qbar[q], 1);
     }
-    mbar_init(&gambar[0], 1);
-    mbar_init(&gambar[1], 1);
     *give_up = 0;
     mbar_fence_init();
   }
@@ -156,7 +182,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
   fence_proxy_async_shared();
   __syncthreads();
 
-  auto flag_timeout = [&](int where) {
+  const int gamma_threads = 32 * (math_warps + 1);  // recurrence warp and math warps meet at the gamma barriers 1 and 2
+  auto flag_timeout = [&](int where) __attribute__((always_inline)) {
     set_status(p.status, DEV_TIMEOUT, where, (long long)blockIdx.x);
     for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
   };
@@ -204,9 +231,10 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
         if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
       }
       // ---- G_b and C_{b-1,b}: sum over the math warps of the cluster ---------------------------------------------
+      bool stop = false;
       if (!mbar_wait_or_give_up(&gbar[q], parity, bp.spin_limit, give_up, true)) {
         if (!*give_up) flag_timeout(2);
-        break;
+        stop = true;
       }
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       float pcorr = 0.0f;   // lane n: sum_m gamma_prev_m C_mn
@@ -232,10 +260,11 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
         __syncwarp();
       }
       // ---- q_b, then p_b = a^B q_b - C^T gamma_{b-1} (b = 0: p = q) -----------------------------------------------
-      if (!mbar_wait_or_give_up(&qbar[q], parity, bp.spin_limit, give_up, true)) {
+      if (!stop && !mbar_wait_or_give_up(&qbar[q], parity, bp.spin_limit, give_up, true)) {
         if (!*give_up) flag_timeout(3);
-        break;
+        stop = true;
       }
+      if (*give_up) stop = true;
       float psum;
       {
         const float* rQ = redQ + (size_t)q * LAG_SLOTS * B + n;
@@ -297,16 +326,18 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
           for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
         }
       }
-      // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}; [8] = 1 - a^nv
+      // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}; [8] = 1 - a^nv; [9] = leave after this block
       float mine = dl_nv;
 #pragma unroll
       for (int m = 0; m < B; ++m) {
         gprev[m] = beta[m] * a_nv;
         if (lane == m) mine = gprev[m];
       }
-      if (lane <= B) gam[(b & 1) * 16 + lane] = mine;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&gambar[b & 1]);  // gamma_b published
+      if (lane == B + 1) mine = stop ? 1.0f : 0.0f;
+      if (lane <= B + 1) gam[(b & 1) * 16 + lane] = mine;
+      if (b & 1) named_bar_arrive(2, gamma_threads);  // gamma_b published
+      else named_bar_arrive(1, gamma_threads);
+      if (stop) break;
     }
     cluster_barrier();  // nobody exits while a peer may still store into its shared memory
     return;
@@ -318,10 +349,10 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
     // the stage's "landed" barrier. A stage is refilled once every math warp has reported that it is done with it.
     const uint32_t copy_bytes = (uint32_t)my_chunks * 16u;
     uint32_t id_next = 0u;
-    auto peek = [&](long long blk) {
+    auto peek = [&](long long blk) __attribute__((always_inline)) {
       if (lane < B && blk < nb) id_next = idx[blk * B + lane];
     };
-    auto request = [&](long long blk, int stg) {
+    auto request = [&](long long blk, int stg) __attribute__((always_inline)) {
       if (blk < nb && blk != bp.drop_block && copy_bytes > 0) {
         if (lane == 0) mbar_arrive_expect_tx(&full[stg], B * copy_bytes);
         __syncwarp();
@@ -385,34 +416,33 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
   const size_t tile_off = (size_t)trow * row_stride + (size_t)mw * 512 + (size_t)(tile >> 1) * 16;
   const int slot = (int)rank * math_warps + mw;
   const uint32_t own_base = (uint32_t)__cvta_generic_to_shared(smem);
-  uint32_t peer_base[8];
-#pragma unroll
-  for (int rr = 0; rr < 8; ++rr) peer_base[rr] = map_shared_rank(smem, (uint32_t)rr < C ? (uint32_t)rr : rank);
-  bool alive = true;  // false once a wait gave up: the warp only walks to the end
+  bool alive = true;  // false once the recurrence warp has published "stop"
 
-  auto wait_rows = [&](long long blk) {
+  auto wait_rows = [&](long long blk) __attribute__((always_inline)) {
     if (my_chunks > 0 && !mbar_wait_or_give_up(&full[blk % S], (uint32_t)((blk / S) & 1), bp.spin_limit, give_up, false)) {
       if (!*give_up) flag_timeout(1);
-      alive = false;
     }
   };
   // [G_new ; C_old,new] over this warp's columns -> table of block blk_new in every CTA of the cluster
-  auto gram_pass = [&](long long blk_new, long long blk_old) {
+  auto gram_pass = [&](long long blk_new, long long blk_old) __attribute__((always_inline)) {
     const unsigned char* src = ring + (size_t)(((tile & 1) ? blk_old : blk_new) % S) * B * row_stride + tile_off;
+    // eight independent accumulators (the instruction's latency is a few hundred cycles), two rounds of eight
+    // 16-column steps; the operand tiles are loaded four at a time
     float acc[8][4];
 #pragma unroll
     for (int a = 0; a < 8; ++a)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][e] = 0.0f;
 #pragma unroll
-    for (int round = 0; round < 2; ++round) {
-      uint32_t q[8][4];
+    for (int round = 0; round < 4; ++round) {
+      uint32_t q[4][4];
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
-        if (round * 8 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 8 + a) * 32);
+      for (int a = 0; a < 4; ++a)
+        if (round * 4 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 4 + a) * 32);
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
-        if (round * 8 + a < ksteps) mma_bf16_m16n8k16(acc[a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
+      for (int a = 0; a < 4; ++a)
+        if (round * 4 + a < ksteps)
+          mma_bf16_m16n8k16(acc[(round & 1) * 4 + a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
     }
 #pragma unroll
     for (int h = 4; h >= 1; h >>= 1)
@@ -424,17 +454,15 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
     const int q = (int)(blk_new & (LAG_DEPTH - 1));
     const uint32_t og = (uint32_t)__cvta_generic_to_shared(redGC + ((size_t)q * LAG_SLOTS + slot) * LAG_GC_VALS + lane * 2) - own_base;
     const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&gbar[q]) - own_base;
-#pragma unroll
-    for (int rr = 0; rr < 8; ++rr) {
-      if ((uint32_t)rr < C) {
-        st_async_f32x2(peer_base[rr] + og, acc[0][0], acc[0][1], peer_base[rr] + ob);
-        st_async_f32x2(peer_base[rr] + og + 64 * (uint32_t)sizeof(float), acc[0][2], acc[0][3], peer_base[rr] + ob);
-      }
+    for (uint32_t rr = 0; rr < C; ++rr) {
+      const uint32_t peer = map_shared_rank(smem, rr);  // the same offsets apply inside every CTA's window
+      st_async_f32x2(peer + og, acc[0][0], acc[0][1], peer + ob);
+      st_async_f32x2(peer + og + 64 * (uint32_t)sizeof(float), acc[0][2], acc[0][3], peer + ob);
     }
   };
   // this thread's columns of the rows of block blk into registers; q = w . x over them, summed over the warp,
   // -> table of block blk in every CTA of the cluster
-  auto q_pass = [&](long long blk, uint4 (&raw)[B]) {
+  auto q_pass = [&](long long blk, uint4 (&raw)[B]) __attribute__((always_inline)) {
     const unsigned char* stage = ring + (size_t)(blk % S) * B * row_stride;
 #pragma unroll
     for (int m = 0; m < B; ++m)
@@ -454,13 +482,14 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
     const uint32_t oq = (uint32_t)__cvta_generic_to_shared(redQ + ((size_t)q * LAG_SLOTS + slot) * B + (lane >> 2)) - own_base;
     const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&qbar[q]) - own_base;
     if ((lane & 3) == 0) {
-#pragma unroll
-      for (int rr = 0; rr < 8; ++rr)
-        if ((uint32_t)rr < C) st_async_f32(peer_base[rr] + oq, qtot, peer_base[rr] + ob);
+      for (uint32_t rr = 0; rr < C; ++rr) {
+        const uint32_t peer = map_shared_rank(smem, rr);
+        st_async_f32(peer + oq, qtot, peer + ob);
+      }
     }
   };
   // w <- w - (1 - a^nv) w - sum_m gamma_m x_m with the rows of block i held in raw
-  auto update = [&](long long i, const uint4 (&raw)[B]) {
+  auto update = [&](long long i, const uint4 (&raw)[B]) __attribute__((always_inline)) {
     const float* g = gam + (i & 1) * 16;
     float2 ngm2[B];
 #pragma unroll
@@ -479,22 +508,24 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
     }
   };
   // iteration i; raw holds the rows of block i on entry and those of block i + 2 on exit
-  auto iteration = [&](long long i, uint4 (&raw)[B]) {
+  auto iteration = [&](long long i, uint4 (&raw)[B]) __attribute__((always_inline)) {
     if (i + 1 < nb) {
       wait_rows(i + 1);
-      if (alive) gram_pass(i + 1, i);
+      gram_pass(i + 1, i);
     }
     // nothing in shared memory of block i is read after this point
     __syncwarp();
     if (lane == 0) mbar_arrive(&fre[i % S]);
-    if (alive && !mbar_wait_or_give_up(&gambar[i & 1], (uint32_t)((i >> 1) & 1), bp.spin_limit, give_up, false)) {
-      if (!*give_up) flag_timeout(5);
+    if (i & 1) named_bar_sync(2, gamma_threads);  // gamma_i and the decision are in gam
+    else named_bar_sync(1, gamma_threads);
+    if (gam[(i & 1) * 16 + B + 1] != 0.0f) {
       alive = false;
+      return;
     }
-    if (alive) update(i, raw);
+    update(i, raw);
     if (i + 2 < nb) {
       wait_rows(i + 2);
-      if (alive) q_pass(i + 2, raw);
+      q_pass(i + 2, raw);
     }
   };
 
@@ -505,14 +536,12 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
   for (int m = 0; m < B; ++m) raw_even[m] = raw_odd[m] = make_uint4(0u, 0u, 0u, 0u);
   if (nb > 0) {
     wait_rows(0);
-    if (alive) {
-      q_pass(0, raw_even);  // p of block 0
-      gram_pass(0, 0);      // G of block 0 (the other half of the table is not used for block 0)
-    }
+    q_pass(0, raw_even);  // p of block 0
+    gram_pass(0, 0);      // G of block 0 (the other half of the table is not used for block 0)
   }
   if (nb > 1) {
     wait_rows(1);
-    if (alive) q_pass(1, raw_odd);  // q of block 1 against the starting model
+    q_pass(1, raw_odd);  // q of block 1 against the starting model
   }
   for (long long i = 0; i < nb && alive; i += 2) {
     iteration(i, raw_even);

@@ -519,9 +519,10 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if (chunks < 1) return false;
   int C = c->opt_cluster;
   if (C <= 0) {
-    // about two CTAs per SM over the whole grid, at least two full warps of chunks per CTA
+    // wide rows are split four ways, with at least two full warps of chunks per CTA (measured on k = 128, d = 4096:
+    // 11.3 ms with two CTAs per chain, 10.5 ms with four, 12.0 ms with eight)
     C = 1;
-    while (C < 8 && (long long)c->k * (C * 2) <= 2 * 148 && chunks / (C * 2) >= 64) C *= 2;
+    while (C < 4 && chunks / (C * 2) >= 64) C *= 2;
     while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;  // a CTA takes at most 8 math warps of 32 chunks
   }
   if (C != 1 && C != 2 && C != 4 && C != 8) return false;
@@ -529,9 +530,10 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
   const long long mw = (cpc + 31) / 32;
   if (mw > 8 || mw * C > MMA_SLOTS) return false;
-  // ring depth: as deep as asked for (default 4) while two CTAs still share an SM; else one CTA per SM
+  // ring depth: as deep as asked for (default 2: a stage is free again as soon as its block has been through the
+  // tensor-core pass, and a shallow ring lets more CTAs share an SM) while two CTAs still share an SM; else one per SM
   const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
-  int want = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
+  int want = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
   int stages = want;
   while (stages > 2 && MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) --stages;
   if (MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) {
@@ -741,9 +743,12 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
   int wR = 0, wstages = 0, wwarps = 0;
   const bool block_warp_ok = block_warp_kernel_fits<XT>(c, aligned, &wR, &wstages, &wwarps);
+  ClusterShape mma_shape;
+  const bool mma_ok = sizeof(XT) == 2 && mma_kernel_fits(c, aligned, &mma_shape);
   if (variant == 0) {
     if (!aligned) variant = 1;
     else if (chunks <= 64) variant = block_warp_ok ? 5 : 3;
+    else if (sizeof(XT) == 2 && chunks >= 256 && mma_ok) variant = 8;  // wide bf16 rows: tensor-core cluster kernel
     else if (block_ok) variant = 4;
     else variant = (chunks > 512 * 4) ? 1 : 2;
   }

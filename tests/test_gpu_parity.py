@@ -481,6 +481,17 @@ def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
         b.check()
 
 
+def test_tensor_core_cluster_kernel_is_the_default_for_wide_bf16_rows(P):
+    wl = wi.config3(k=4, d=2048, m=64, n_lo=60, n_hi=120).to("cuda")
+    with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
+        a.run_workload(wl)
+        b.set_option("dense_variant", 8)
+        b.run_workload(wl)
+        np.testing.assert_array_equal(a.get_models().cpu().numpy(), b.get_models().cpu().numpy())
+        a.check()
+        b.check()
+
+
 # ---- degenerate cases -----------------------------------------------------------------------------------
 def test_nodes_without_work_keep_w0(P):
     wl = wi.config1(k=4, d=64, m=64, n_steps=(120, 0, 30, 0))
