@@ -48,8 +48,8 @@ struct MmaSmem {
     w3 = ring + (size_t)stages * BLK_B * row_stride;                // w_hi, w_mid, w_lo, one zero row
     redG = w3 + 4 * row_stride;                                     // [2][slots][64]
     redP = redG + 2 * (size_t)MMA_SLOTS * MMA_G_VALS * sizeof(float);  // [2][slots][32]
-    totG = redP + 2 * (size_t)MMA_SLOTS * MMA_P_VALS * sizeof(float);  // [64]
-    gam = totG + 64 * sizeof(float);                                // gamma_0..7, 1 - a^nv, stop
+    totG = redP + 2 * (size_t)MMA_SLOTS * MMA_P_VALS * sizeof(float);  // [64] G, [32] parts of p
+    gam = totG + 96 * sizeof(float);                                // gamma_0..7, 1 - a^nv, stop
     tab = gam + 16 * sizeof(float);                                 // [48]
     jet = tab + 3 * 16 * sizeof(float);                             // [8] float4
     bars = jet + 8 * 4 * sizeof(float);                             // ring barriers [8]
@@ -87,7 +87,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 template <int LOSS>
-__global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const ClusterParams cp) {
+__global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const ClusterParams cp) {
   constexpr int B = BLK_B;
   extern __shared__ __align__(16) unsigned char smem[];
   const BlockParams& bp = cp.b;
@@ -203,16 +203,21 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
       const float* rG = redG + (size_t)q * MMA_SLOTS * MMA_G_VALS;
       const float* rP = redP + (size_t)q * MMA_SLOTS * MMA_P_VALS;
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
+      float psum;           // lane l: p of sample l & 7
       {
-        float g0[MMA_SLOTS], g1[MMA_SLOTS];
+        // one pass over the slots with 16-byte loads: lanes 0..15 add four consecutive entries of G each, lanes
+        // 16..23 four of the parts of p
+        if (lane < 24) {
+          const float* base = lane < 16 ? rG + lane * 4 : rP + (lane & 7) * 4;
+          const int stride = lane < 16 ? MMA_G_VALS : MMA_P_VALS;
+          float4 s4 = *(const float4*)base;
 #pragma unroll
-        for (int w = 0; w < MMA_SLOTS; ++w) { g0[w] = rG[w * 64 + lane]; g1[w] = rG[w * 64 + 32 + lane]; }
-#pragma unroll
-        for (int h = MMA_SLOTS / 2; h >= 1; h >>= 1)
-#pragma unroll
-          for (int w = 0; w < h; ++w) { g0[w] += g0[w + h]; g1[w] += g1[w + h]; }
-        totG[lane] = g0[0];
-        totG[32 + lane] = g1[0];
+          for (int w = 1; w < MMA_SLOTS; ++w) {
+            const float4 v = *(const float4*)(base + w * stride);
+            s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
+          }
+          ((float4*)totG)[lane] = s4;
+        }
         __syncwarp();
 #pragma unroll
         for (int n2 = 1; n2 < B; ++n2) {
@@ -221,20 +226,9 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
 #pragma unroll
           for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] = row[m] * sc[n2];
         }
+        // rows 8..10 of the accumulator: w_hi . x_n, w_mid . x_n, w_lo . x_n; small terms first
+        psum = (totG[64 + 16 + n] + totG[64 + 8 + n]) + totG[64 + n];
         __syncwarp();
-      }
-      float psum;
-      {
-        float pp[MMA_SLOTS];
-#pragma unroll
-        for (int w = 0; w < MMA_SLOTS; ++w) pp[w] = rP[w * MMA_P_VALS + lane];
-#pragma unroll
-        for (int h = MMA_SLOTS / 2; h >= 1; h >>= 1)
-#pragma unroll
-          for (int w = 0; w < h; ++w) pp[w] += pp[w + h];
-        // lanes 0..7: w_hi . x_n, 8..15: w_mid . x_n, 16..23: w_lo . x_n (24..31: zero); small terms first
-        const float mid = __shfl_down_sync(0xffffffffu, pp[0], 8), lo = __shfl_down_sync(0xffffffffu, pp[0], 16);
-        psum = (lo + mid) + pp[0];  // lanes 0..7: p_n
       }
       float t[B], beta[B];
 #pragma unroll
@@ -409,27 +403,29 @@ __global__ void __launch_bounds__(64 + 32 * 8, 2) chain_mma_kernel(const Cluster
     }
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
     // ---- [G_b ; p_b parts] over this warp's columns ------------------------------------------------------------
-    // eight independent accumulators (the instruction's latency is long), two rounds of eight 16-column steps
-    float acc[8][4];
+    // one accumulator per 16-column step (the instruction's latency is several hundred cycles: no step waits for
+    // another); the operand tiles are loaded four at a time
+    float acc[16][4];
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
+    for (int a = 0; a < 16; ++a)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][e] = 0.0f;
     {
       const unsigned char* src = (tile & 1) ? w_src : stage + x_off;
 #pragma unroll
-      for (int round = 0; round < 2; ++round) {
-        uint32_t q[8][4];
+      for (int round = 0; round < 4; ++round) {
+        uint32_t q[4][4];
 #pragma unroll
-        for (int a = 0; a < 8; ++a)
-          if (round * 8 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 8 + a) * 32);
+        for (int a = 0; a < 4; ++a)
+          if (round * 4 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 4 + a) * 32);
 #pragma unroll
-        for (int a = 0; a < 8; ++a)
-          if (round * 8 + a < ksteps) mma_bf16_m16n8k16(acc[a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
+        for (int a = 0; a < 4; ++a)
+          if (round * 4 + a < ksteps)
+            mma_bf16_m16n8k16(acc[round * 4 + a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
       }
     }
 #pragma unroll
-    for (int h = 4; h >= 1; h >>= 1)
+    for (int h = 8; h >= 1; h >>= 1)
 #pragma unroll
       for (int a = 0; a < h; ++a)
 #pragma unroll

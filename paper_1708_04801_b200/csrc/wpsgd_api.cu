@@ -519,11 +519,11 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if (chunks < 1) return false;
   int C = c->opt_cluster;
   if (C <= 0) {
-    // wide rows are split four ways, with at least two full warps of chunks per CTA (measured on k = 128, d = 4096:
-    // 11.3 ms with two CTAs per chain, 10.5 ms with four, 12.0 ms with eight)
+    // as few CTAs per chain as the row width allows (a CTA takes at most 8 math warps of 32 chunks): the kernel runs
+    // one CTA per SM, and what a wider cluster gains in the tensor-core pass it loses in chains running at the same
+    // time (measured on k = 128, d = 4096: 7.95 ms with two CTAs per chain, 9.9 ms with four, 14.0 ms with eight)
     C = 1;
-    while (C < 4 && chunks / (C * 2) >= 64) C *= 2;
-    while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;  // a CTA takes at most 8 math warps of 32 chunks
+    while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;
   }
   if (C != 1 && C != 2 && C != 4 && C != 8) return false;
   const long long cpc = (chunks + C - 1) / C;
