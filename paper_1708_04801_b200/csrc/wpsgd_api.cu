@@ -13,6 +13,7 @@
 #include "chain_block.cuh"
 #include "chain_cluster.cuh"
 #include "chain_csr.cuh"
+#include "chain_gram.cuh"
 #include "chain_lag.cuh"
 #include "chain_mma.cuh"
 #include "chain_tc.cuh"
@@ -659,6 +660,48 @@ wpsgd_status launch_lag(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   }
 }
 
+// ---- blocked kernel with Gram warps (one CTA per node, rows of up to 256 chunks) ---------------------------------------
+template <typename XT>
+bool gram_kernel_fits(const wpsgd_ctx* c, bool aligned, int* math_warps_out, int* stages_out) {
+  constexpr int V = XVec<XT>::V;
+  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / V;
+  if (chunks < 1 || chunks > 32 * GRAM_MAX_MATH_WARPS) return false;
+  const size_t row_bytes = (size_t)c->d * sizeof(XT);
+  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
+  while (stages >= 2 && GramSmem(stages, row_bytes).total > kSmemBudget) --stages;
+  if (stages < 2) return false;
+  *math_warps_out = (int)((chunks + 31) / 32);
+  *stages_out = stages;
+  return true;
+}
+
+template <typename XT>
+wpsgd_status launch_gram(wpsgd_ctx* c, const ChainParams& p, int math_warps, int stages) {
+  BlockParams bp;
+  bp.c = p;
+  bp.stages = stages;
+  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  bp.spin_limit = c->opt_spin_limit;
+  bp.drop_block = c->opt_drop_block;
+  bp.group_order = nullptr;
+  const size_t smem = GramSmem(stages, (size_t)c->d * sizeof(XT)).total;
+  const int threads = 64 + 32 * math_warps + 32 * ((math_warps + 1) / 2);  // math warps and one Gram warp per 64 chunks
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<c->k, threads, smem, c->stream>>>(bp);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_gram_kernel<XT, LOSS_HINGE>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_gram_kernel<XT, LOSS_LOGISTIC>);
+    default: return go(chain_gram_kernel<XT, LOSS_SQUARED>);
+  }
+}
+
 // blocked kernel, one warp per node (small d)
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
@@ -758,6 +801,13 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
+  }
+  if (variant == 10) {
+    int gmw = 0, gstages = 0;
+    if (!gram_kernel_fits<XT>(c, aligned, &gmw, &gstages))
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "Gram-warp kernel needs 16-byte aligned rows of at most 256 chunks, a constant step size and eta*lambda <= 0.25");
+    return launch_gram<XT>(c, p, gmw, gstages);
   }
   if (variant == 9) {
     ClusterShape sh;
@@ -980,7 +1030,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 9) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..9");
+    if (value < 0 || value > 10) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..10");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");
