@@ -78,7 +78,13 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
  * mix(R ^ key) = multiply 0x85EBCA6B, xor-shift 13, multiply 0xC2B2AE35, xor-shift 16, masked to half the bits.
  * Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
  * with register-held model, 3 warp per node, 4 blocked kernel: 8 samples per synchronisation, CTA per node; 5 the same with a warp per node; 6 the blocked kernel for bf16 rows with the Gram products on
- * tcgen05 tensor cores, 64 samples at a time (kept for comparison: measured slower than 4 on B200)), "prefetch" (rows in
+ * tcgen05 tensor cores, 64 samples at a time (kept for comparison: measured slower than 4 on B200); 7 the blocked form with the
+ * columns of a node split over a thread-block cluster, packed fp32 FMAs; 8 the same split for bf16 rows with the Gram block
+ * and the margins of a block from mma.sync tensor-core instructions, the fp32 model entering as three bf16 rows (what 0
+ * picks for aligned bf16 rows of 2048 to 4096 columns); 9 bf16 rows, margins taken one block behind the model ("lagged" form);
+ * 10 one CTA per node with the Gram block formed by warps of its own (rows of up to 256 16-byte chunks)), "cluster" (CTAs
+ * per node of variants 7, 8, 9: 0 = chosen from d, else 1, 2, 4 or 8), "chunks_per_thread" (variant 7: 16-byte chunks of a
+ * row per math thread, 0 = chosen, 1 or 2), "prefetch" (rows in
  * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "stages" (blocks of 8 rows in the shared-memory ring of the blocked kernel; 0 = as many as fit, up to 4), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
  * (polls after which a device-side wait gives up), "tc_gram" (1: bf16 rows take the 8x8 Gram block of the blocked kernel from mma.sync tensor-core
  * instructions instead of FFMA; same result up to summation order), "test_drop_block" (test hook of the bounded wait: the rows of
