@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--rho", type=float, default=4.0, help="speed ratio of workload 5")
     ap.add_argument("--small", action="store_true", help="scaled-down copy of the workload (profiling captures)")
     ap.add_argument("--rows", type=int, default=0, help="rows per node override (smaller device footprint for profiler captures)")
-    ap.add_argument("--also", default="3,5", help="further workloads measured after the main one at 1 GPU and reported "
+    ap.add_argument("--also", default="3,5,4", help="further workloads measured after the main one at 1 GPU and reported "
                     "under other_workloads (device-resident timing only); empty to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="name=value passed to wpsgd_set_option")

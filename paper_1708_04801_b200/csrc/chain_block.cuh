@@ -114,6 +114,26 @@ __device__ __forceinline__ void widen_quad<__nv_bfloat16>(const uint4& raw, int 
   f[2] = __uint_as_float(b << 16); f[3] = __uint_as_float(b & 0xffff0000u);
 }
 
+// The columns of a 16-byte chunk as pairs of fp32 (the operand form of the packed FMA).
+template <typename XT>
+struct XPairs;
+template <>
+struct XPairs<float> {
+  static constexpr int NP = 2;
+  __device__ __forceinline__ static float2 get(const uint4& raw, int i) {
+    return i == 0 ? make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y))
+                  : make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
+  }
+};
+template <>
+struct XPairs<__nv_bfloat16> {
+  static constexpr int NP = 4;
+  __device__ __forceinline__ static float2 get(const uint4& raw, int i) {
+    const uint32_t u = i == 0 ? raw.x : (i == 1 ? raw.y : (i == 2 ? raw.z : raw.w));
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+  }
+};
+
 // Sum of each of 32 per-lane values over the warp; afterwards lane l holds the total of value l.
 // 31 shuffles: in every round a lane hands half of its values to its partner and keeps the other half.
 __device__ __forceinline__ float warp_transpose_sum32(float (&v)[32]) {
@@ -835,29 +855,37 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
     prefetch_block(b + S, st, id_lo, id_hi);
     load_ids(b + 1 + S, id_lo, id_hi);
     // ---- G_b and p_b in one pass -----------------------------------------------------------------------
+    // packed two-wide fp32 FMAs: even and odd columns accumulate side by side and are added at the end
     float acc[32], accp[B];
+    {
+      constexpr int NP = XPairs<XT>::NP;
+      float2 acc2[BLK_PAIRS], accp2[B];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+      for (int i = 0; i < BLK_PAIRS; ++i) acc2[i] = make_float2(0.0f, 0.0f);
 #pragma unroll
-    for (int m = 0; m < B; ++m) accp[m] = 0.0f;
+      for (int m = 0; m < B; ++m) accp2[m] = make_float2(0.0f, 0.0f);
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
+      for (int r = 0; r < R; ++r) {
 #pragma unroll
-      for (int q = 0; q < QV; ++q) {
-        float x[B][4];
+        for (int i = 0; i < NP; ++i) {
+          float2 x2[B];
 #pragma unroll
-        for (int m = 0; m < B; ++m) widen_quad<XT>(raw[r][m], q, x[m]);
+          for (int m = 0; m < B; ++m) x2[m] = XPairs<XT>::get(raw[r][m], i);
 #pragma unroll
-        for (int n2 = 1; n2 < B; ++n2)
+          for (int n2 = 1; n2 < B; ++n2)
 #pragma unroll
-          for (int m = 0; m < n2; ++m)
+            for (int m = 0; m < n2; ++m) acc2[n2 * (n2 - 1) / 2 + m] = __ffma2_rn(x2[m], x2[n2], acc2[n2 * (n2 - 1) / 2 + m]);
+          const float2 wp = make_float2(w[r][2 * i], w[r][2 * i + 1]);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) acc[n2 * (n2 - 1) / 2 + m] = fmaf(x[m][e], x[n2][e], acc[n2 * (n2 - 1) / 2 + m]);
-#pragma unroll
-        for (int m = 0; m < B; ++m)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) accp[m] = fmaf(w[r][q * 4 + e], x[m][e], accp[m]);
+          for (int m = 0; m < B; ++m) accp2[m] = __ffma2_rn(wp, x2[m], accp2[m]);
+        }
       }
+#pragma unroll
+      for (int i = 0; i < BLK_PAIRS; ++i) acc[i] = acc2[i].x + acc2[i].y;
+#pragma unroll
+      for (int i = BLK_PAIRS; i < 32; ++i) acc[i] = 0.0f;
+#pragma unroll
+      for (int m = 0; m < B; ++m) accp[m] = accp2[m].x + accp2[m].y;
     }
     const float ptot = warp_transpose_sum8(accp);   // every lane: total of p_{lane >> 2}
     const float gtot = warp_transpose_sum32(acc);   // lane l: total of Gram entry l
@@ -945,19 +973,25 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
       }
     }
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m,  gamma_m = beta_m a^nv ----------------------------------
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-#pragma unroll
-      for (int v = 0; v < V; ++v) w[r][v] = fmaf(-dl, w[r][v], w[r][v]);
+    {
+      constexpr int NP = XPairs<XT>::NP;
+      float2 ngm2[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) {
-        const float gm = beta[m] * a_nv;
+        const float gm = -(beta[m] * a_nv);
+        ngm2[m] = make_float2(gm, gm);
+      }
+      const float2 ndl2 = make_float2(-dl, -dl);
 #pragma unroll
-        for (int q = 0; q < QV; ++q) {
-          float x[4];
-          widen_quad<XT>(raw[r][m], q, x);
+      for (int r = 0; r < R; ++r) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) w[r][q * 4 + e] = fmaf(-gm, x[e], w[r][q * 4 + e]);
+        for (int i = 0; i < NP; ++i) {
+          float2 wv = make_float2(w[r][2 * i], w[r][2 * i + 1]);
+          wv = __ffma2_rn(ndl2, wv, wv);
+#pragma unroll
+          for (int m = 0; m < B; ++m) wv = __ffma2_rn(ngm2[m], XPairs<XT>::get(raw[r][m], i), wv);
+          w[r][2 * i] = wv.x;
+          w[r][2 * i + 1] = wv.y;
         }
       }
     }

@@ -61,26 +61,6 @@ __device__ __forceinline__ void st_shared_cluster(uint32_t addr, int v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// The columns of a 16-byte chunk as pairs of fp32 (the operand form of the packed FMA).
-template <typename XT>
-struct XPairs;
-template <>
-struct XPairs<float> {
-  static constexpr int NP = 2;
-  __device__ __forceinline__ static float2 get(const uint4& raw, int i) {
-    return i == 0 ? make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y))
-                  : make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
-  }
-};
-template <>
-struct XPairs<__nv_bfloat16> {
-  static constexpr int NP = 4;
-  __device__ __forceinline__ static float2 get(const uint4& raw, int i) {
-    const uint32_t u = i == 0 ? raw.x : (i == 1 ? raw.y : (i == 2 ? raw.z : raw.w));
-    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
-  }
-};
-
 constexpr int CL_MAX_SLOTS = 16;  // math warps of a whole cluster
 
 struct ClusterSmem {

@@ -4,20 +4,20 @@
 // With few nodes a chain is bound by the dependent loop of a block: model update -> p = X_b w -> 8-step recurrence ->
 // model update. The Gram block G_b = X_b X_b^T does not depend on the model; in chain_block_kernel the math warps
 // form it while the recurrence runs, but it takes them about twice as long as the recurrence, so it ends up on the
-// path. Here the math warps only keep the model (p and update), and "Gram warps" form G_{b+1} between the two
-// barriers of block b: Gram warp c takes the 28 entries over the c-th group of 64 16-byte chunks (two chunks per
-// lane). W math warps (32 chunks each) and ceil(chunks / 64) Gram warps: 14 warps for 256 chunks, which leaves every
-// thread 128 registers (the recurrence warp needs about 120; with fewer it spills into its dependent chain).
+// path. Here the math warps only keep the model (p and update), and "Gram warps" form the Gram block two blocks
+// ahead, beside the math warps' part of the loop, so that the recurrence has the SM to itself: Gram warp c takes the
+// 28 entries over the c-th group of 64 16-byte chunks (two chunks per lane). W math warps (32 chunks each) and ceil(chunks / 64) Gram warps: 14 warps for
+// 256 chunks, which leaves every thread 128 registers (the recurrence warp needs about 120).
 //
 //                math warps                   Gram warps                           recurrence warp
-//                p_b partials -> smem         -                                    sum G_b partials (last round)
+//                w <- w - (1-a^B) w - ...     rows of block b+1: G_{b+1} partials   labels, constants of block b,
+//                rows of block b -> regs      -> smem (buffer (b+1) & 1)           sum G_b partials (buffer b & 1)
+//                p_b partials -> smem
 //                ------------------------------ barrier 1 ---------------------------------------------------
-//                -                            rows of block b+1: half of the       sum p_b, recurrence, gamma -> smem
-//                                             G_{b+1} partials -> smem
+//                -                            -                                    sum p_b, recurrence, gamma -> smem
 //                ------------------------------ barrier 2 ---------------------------------------------------
-//                w <- w - (1-a^B) w - sum gamma_m x_m;  rows of block b+1 -> registers
 // The copy warp (warp 1) requests rows with bulk asynchronous copies into a ring of stages (never multicast); the stage
-// of block b is refilled after barrier 1 of block b, when the math warps hold its rows in registers. Waits on arriving
+// of block b is refilled after barrier 1 of block b, when the math warps hold its rows in registers and its Gram block is long done. Waits on arriving
 // rows are bounded; a wait that runs out is flagged before a barrier and read by every warp right after barrier 2.
 #pragma once
 
@@ -32,8 +32,8 @@ struct GramSmem {
   size_t ring, redG, redP, totG, gam, tab, jet, bars, flag, total;
   __host__ __device__ GramSmem(int stages, size_t row_bytes) {
     ring = 0;
-    redG = ring + (size_t)stages * BLK_B * row_bytes;                          // [groups][32]
-    redP = redG + (size_t)GRAM_MAX_GROUPS * 32 * sizeof(float);                // [W][8]
+    redG = ring + (size_t)stages * BLK_B * row_bytes;                          // [2][groups][32]
+    redP = redG + 2 * (size_t)GRAM_MAX_GROUPS * 32 * sizeof(float);            // [W][8]
     totG = redP + (size_t)GRAM_MAX_MATH_WARPS * BLK_B * sizeof(float);         // [32]
     gam = totG + 32 * sizeof(float);                                           // [16]
     tab = gam + 16 * sizeof(float);                                            // [48]
@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(64 + 32 * GRAM_MAX_MATH_WARPS + 32 * GRAM_MAX_
     mbar_fence_init();
   }
   // partial-sum slots that no warp writes stay zero
-  for (int i = threadIdx.x; i < GRAM_MAX_GROUPS * 32; i += blockDim.x) redG[i] = 0.0f;
+  for (int i = threadIdx.x; i < 2 * GRAM_MAX_GROUPS * 32; i += blockDim.x) redG[i] = 0.0f;
   for (int i = threadIdx.x; i < GRAM_MAX_MATH_WARPS * B; i += blockDim.x) redP[i] = 0.0f;
   __syncthreads();  // tables and barriers are set up
 
@@ -165,12 +165,13 @@ __global__ void __launch_bounds__(64 + 32 * GRAM_MAX_MATH_WARPS + 32 * GRAM_MAX_
         }
         if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
       }
-      // G_b: lane l adds entry l over the Gram warps (they finished it during the previous block)
+      // G_b: lane l adds entry l over the Gram warps (they finished it before barrier 1 of the previous block)
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       {
-        float g = redG[lane];
+        const float* rG = redG + (size_t)(b & 1) * GRAM_MAX_GROUPS * 32;
+        float g = rG[lane];
 #pragma unroll
-        for (int w = 1; w < GRAM_MAX_GROUPS; ++w) g += redG[w * 32 + lane];
+        for (int w = 1; w < GRAM_MAX_GROUPS; ++w) g += rG[w * 32 + lane];
         totG[lane] = g;
         __syncwarp();
 #pragma unroll
@@ -301,9 +302,11 @@ __global__ void __launch_bounds__(64 + 32 * GRAM_MAX_MATH_WARPS + 32 * GRAM_MAX_
     // =========================== Gram warps ==============================================================
     const int gw = gram_index;
     const int grp = gw;
-    float* out = redG + (size_t)grp * 32;
-    auto gram_of = [&](int stg) __attribute__((always_inline)) {
-      const unsigned char* stage = ring + (size_t)stg * B * row_bytes;
+    // Gram block of block g (its rows awaited, bounded) -> buffer g & 1
+    auto gram_of = [&](long long g) __attribute__((always_inline)) {
+      wait_rows((int)(g % S), (uint32_t)((g / S) & 1));
+      const unsigned char* stage = ring + (size_t)(g % S) * B * row_bytes;
+      float* out = redG + ((size_t)(g & 1) * GRAM_MAX_GROUPS + grp) * 32;
       float2 acc2[BLK_PAIRS];
 #pragma unroll
       for (int k = 0; k < BLK_PAIRS; ++k) acc2[k] = make_float2(0.0f, 0.0f);
@@ -324,22 +327,14 @@ __global__ void __launch_bounds__(64 + 32 * GRAM_MAX_MATH_WARPS + 32 * GRAM_MAX_
       for (int k = BLK_PAIRS; k < 32; ++k) part[k] = 0.0f;
       out[lane] = warp_transpose_sum32(part);  // lane l: entry l over the warp's columns
     };
-    if (nb > 0) {
-      wait_rows(0, 0u);
-      gram_of(0);
-    }
+    if (nb > 0) gram_of(0);
+    if (nb > 1) gram_of(1);
     __syncthreads();  // start-up barrier
-    int st = (S > 1) ? 1 : 0;          // stage of block b + 1 ...
-    uint32_t par = (S > 1) ? 0u : 1u;  // ... and the parity of the barrier phase that brings it
     for (long long b = 0; b < nb; ++b) {
-      __syncthreads();  // barrier 1: the recurrence warp has read the Gram block of block b
-      if (b + 1 < nb) {
-        wait_rows(st, par);
-        gram_of(st);
-      }
+      __syncthreads();  // barrier 1: the recurrence warp has read the Gram block of block b (buffer b & 1)
       __syncthreads();  // barrier 2
       if (*give_up) break;
-      if (++st == S) { st = 0; par ^= 1u; }
+      if (b + 2 < nb) gram_of(b + 2);  // beside the math warps' update and p, done before barrier 1 of block b + 1
     }
     return;
   }
