@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_lag_kernel(const Cluster
   // [G_new ; C_old,new] over this warp's columns -> table of block blk_new in every CTA of the cluster
   auto gram_pass = [&](long long blk_new, long long blk_old) __attribute__((always_inline)) {
     const unsigned char* src = ring + (size_t)(((tile & 1) ? blk_old : blk_new) % S) * B * row_stride + tile_off;
-    // eight independent accumulators (the instruction's latency is a few hundred cycles), two rounds of eight
+    // eight independent accumulators, two rounds of eight
     // 16-column steps; the operand tiles are loaded four at a time
     float acc[8][4];
 #pragma unroll

@@ -11,8 +11,11 @@
 // columns, the accumulator over the warp's 256). Only the update w <- w - (1 - a^B) w - sum_m gamma_m x_m stays on
 // the fp32 pipes (packed two-wide FMAs), followed by re-splitting the thread's 8 model values into the three bf16 rows.
 //
-// Layout. CTA `rank` of a cluster of C owns the 16-byte chunks [rank * cpc, (rank + 1) * cpc) of every row; math warp
-// mw owns chunks [32 mw, 32 mw + 32) of that slice, lane l chunk 32 mw + l (its 8 model values live in registers).
+// Layout. CTA `rank` of a cluster of C owns the 16-byte chunks [rank * cpc, (rank + 1) * cpc) of every row. A lane
+// owns NPL pairs of consecutive columns (NPL = 4: one 16-byte chunk, 8 math warps cover 2048 columns, the default;
+// NPL = 2: half a chunk, 16 math warps, which halves the instruction stream of a math warp but doubles the partial
+// sums the recurrence warp adds, and measured slower), math warp mw the 32 consecutive lane units from 32 mw; the
+// model values live in registers.
 // Warp 0 runs the recurrence, warp 1 requests rows (bulk asynchronous copies into a ring of stages, one barrier per
 // stage, never multicast). Staged rows and the three model rows have a stride of slice + 16 bytes, which keeps the
 // 8 x 8 tile loads (ldmatrix) free of bank conflicts; bytes beyond a CTA's slice stay zero.
@@ -35,20 +38,20 @@
 
 namespace wpsgd {
 
-constexpr int MMA_SLOTS = 16;    // math warps of a whole cluster
+constexpr int MMA_SLOTS = 16;    // math warps of a whole cluster (one 16-byte chunk per lane); twice that with half chunks
 constexpr int MMA_G_VALS = 64;   // accumulator rows 0..7
 constexpr int MMA_P_VALS = 32;   // accumulator rows 8..10 (24 used)
 constexpr uint32_t MMA_SLOT_BYTES = (64 + 24) * sizeof(float);  // what one math warp sends to one CTA per block
 
 struct MmaSmem {
   size_t row_stride, ring, w3, redG, redP, totG, gam, tab, jet, bars, pbar, flag, total;
-  __host__ __device__ MmaSmem(int stages, size_t slice_bytes) {
+  __host__ __device__ MmaSmem(int stages, size_t slice_bytes, int slots) {
     row_stride = slice_bytes + 16;
     ring = 0;
     w3 = ring + (size_t)stages * BLK_B * row_stride;                // w_hi, w_mid, w_lo, one zero row
     redG = w3 + 4 * row_stride;                                     // [2][slots][64]
-    redP = redG + 2 * (size_t)MMA_SLOTS * MMA_G_VALS * sizeof(float);  // [2][slots][32]
-    totG = redP + 2 * (size_t)MMA_SLOTS * MMA_P_VALS * sizeof(float);  // [64] G, [32] parts of p
+    redP = redG + 2 * (size_t)slots * MMA_G_VALS * sizeof(float);  // [2][slots][32]
+    totG = redP + 2 * (size_t)slots * MMA_P_VALS * sizeof(float);  // [64] G, [32] parts of p
     gam = totG + 96 * sizeof(float);                                // gamma_0..7, 1 - a^nv, stop
     tab = gam + 16 * sizeof(float);                                 // [48]
     jet = tab + 3 * 16 * sizeof(float);                             // [8] float4
@@ -86,9 +89,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
-template <int LOSS>
-__global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const ClusterParams cp) {
+template <int LOSS, int NPL>
+__global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chain_mma_kernel(const ClusterParams cp) {
   constexpr int B = BLK_B;
+  constexpr int LB = NPL * 4;                     // bytes of a row per lane
+  constexpr int KS = LB;                          // 16-column steps per warp (32 lanes x LB bytes / 32 bytes)
+  constexpr int SLOTS = MMA_SLOTS * (4 / NPL);    // partial-sum slots of the cluster
   extern __shared__ __align__(16) unsigned char smem[];
   const BlockParams& bp = cp.b;
   const ChainParams& p = bp.c;
@@ -105,7 +111,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
   const int my_chunks = (int)(chunk_end > chunk0 ? chunk_end - chunk0 : 0);
   const size_t slice_bytes = (size_t)cp.chunks_per_cta * 16;
   const size_t ld_bytes = (size_t)p.ld * 2;
-  const MmaSmem L(S, slice_bytes);
+  const MmaSmem L(S, slice_bytes, SLOTS);
   const size_t row_stride = L.row_stride;
   unsigned char* ring = smem + L.ring;
   unsigned char* w3 = smem + L.w3;
@@ -200,8 +206,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
         }
       }
       const int stop = *give_up;
-      const float* rG = redG + (size_t)q * MMA_SLOTS * MMA_G_VALS;
-      const float* rP = redP + (size_t)q * MMA_SLOTS * MMA_P_VALS;
+      const float* rG = redG + (size_t)q * SLOTS * MMA_G_VALS;
+      const float* rP = redP + (size_t)q * SLOTS * MMA_P_VALS;
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       float psum;           // lane l: p of sample l & 7
       {
@@ -212,7 +218,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
           const int stride = lane < 16 ? MMA_G_VALS : MMA_P_VALS;
           float4 s4 = *(const float4*)base;
 #pragma unroll
-          for (int w = 1; w < MMA_SLOTS; ++w) {
+          for (int w = 1; w < SLOTS; ++w) {
             const float4 v = *(const float4*)(base + w * stride);
             s4.x += v.x; s4.y += v.y; s4.z += v.z; s4.w += v.w;
           }
@@ -346,36 +352,51 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
 
   // ============================= math warps ==============================================================
   const int mw = warp - 2;
-  const int lc = mw * 32 + lane;  // this thread's chunk within the CTA's slice
-  const bool act = lc < my_chunks;
-  const int warp_chunks = my_chunks - mw * 32 < 0 ? 0 : (my_chunks - mw * 32 > 32 ? 32 : my_chunks - mw * 32);
-  const int ksteps = (warp_chunks + 1) >> 1;  // 16 columns (two chunks) per tensor-core instruction
-  float2 w2[4];
+  const int lc = mw * 32 + lane;  // this thread's unit (LB bytes of a row) within the CTA's slice
+  const int my_units = my_chunks * (16 / LB);
+  const bool act = lc < my_units;
+  const int warp_units = my_units - mw * 32 < 0 ? 0 : (my_units - mw * 32 > 32 ? 32 : my_units - mw * 32);
+  const int ksteps = (warp_units * LB + 31) / 32;  // 16 columns (32 bytes) per tensor-core instruction
+  float2 w2[NPL];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) w2[i] = make_float2(0.0f, 0.0f);
+  for (int i = 0; i < NPL; ++i) w2[i] = make_float2(0.0f, 0.0f);
   if (act) {
-    const long long c0 = (chunk0 + lc) * 8;
+    const long long c0 = chunk0 * 8 + (long long)lc * (2 * NPL);
     const float* src = p.resume ? (p.W + (size_t)j * d + c0) : (p.w0 ? p.w0 + c0 : nullptr);
     if (src) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) w2[i] = make_float2(src[2 * i], src[2 * i + 1]);
+      for (int i = 0; i < NPL; ++i) w2[i] = make_float2(src[2 * i], src[2 * i + 1]);
     }
   }
-  // the thread's 8 model values as three bf16 rows: w = hi + mid + lo (each remainder is exact in fp32)
-  auto publish_model = [&]() {
+  // LB bytes of shared memory as NPL words
+  auto load_words = [&](const unsigned char* ptr, uint32_t (&wd)[NPL]) __attribute__((always_inline)) {
+    if (NPL == 4) {
+      const uint4 v = *(const uint4*)ptr;
+      wd[0] = v.x; wd[1] = v.y; wd[NPL - 2] = v.z; wd[NPL - 1] = v.w;
+    } else {
+      const uint2 v = *(const uint2*)ptr;
+      wd[0] = v.x; wd[1] = v.y;
+    }
+  };
+  auto store_words = [&](unsigned char* ptr, const uint32_t (&wd)[NPL]) __attribute__((always_inline)) {
+    if (NPL == 4) *(uint4*)ptr = make_uint4(wd[0], wd[1], wd[NPL - 2], wd[NPL - 1]);
+    else *(uint2*)ptr = make_uint2(wd[0], wd[1]);
+  };
+  // the thread's model values as three bf16 rows: w = hi + mid + lo (each remainder is exact in fp32)
+  auto publish_model = [&]() __attribute__((always_inline)) {
     if (act) {
-      uint32_t hi[4], mid[4], lo[4];
+      uint32_t hi[NPL], mid[NPL], lo[NPL];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < NPL; ++i) {
         hi[i] = pack_bf16x2(w2[i].x, w2[i].y);
         const float rx = w2[i].x - __uint_as_float(hi[i] << 16), ry = w2[i].y - __uint_as_float(hi[i] & 0xffff0000u);
         mid[i] = pack_bf16x2(rx, ry);
         const float sx = rx - __uint_as_float(mid[i] << 16), sy = ry - __uint_as_float(mid[i] & 0xffff0000u);
         lo[i] = pack_bf16x2(sx, sy);
       }
-      *(uint4*)(w3 + 0 * row_stride + (size_t)lc * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      *(uint4*)(w3 + 1 * row_stride + (size_t)lc * 16) = make_uint4(mid[0], mid[1], mid[2], mid[3]);
-      *(uint4*)(w3 + 2 * row_stride + (size_t)lc * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      store_words(w3 + 0 * row_stride + (size_t)lc * LB, hi);
+      store_words(w3 + 1 * row_stride + (size_t)lc * LB, mid);
+      store_words(w3 + 2 * row_stride + (size_t)lc * LB, lo);
     }
     __syncwarp();
   };
@@ -383,7 +404,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
   // tile addresses of the tensor-core operand loads: lanes 8i..8i+7 give the 8 row addresses of tile i; tiles 0 and 2
   // are the staged rows (columns +0 and +8), tiles 1 and 3 the model rows (hi, mid, lo, then the zero row)
   const int tile = lane >> 3, trow = lane & 7;
-  const size_t tile_col_bytes = (size_t)mw * 512 + (size_t)(tile >> 1) * 16;
+  const size_t tile_col_bytes = (size_t)mw * (32 * LB) + (size_t)(tile >> 1) * 16;
   const size_t x_off = (size_t)trow * row_stride + tile_col_bytes;
   const unsigned char* w_src = w3 + (size_t)(trow < 3 ? trow : 3) * row_stride + tile_col_bytes;
   const int slot = (int)rank * math_warps + mw;
@@ -403,17 +424,17 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
     }
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
     // ---- [G_b ; p_b parts] over this warp's columns ------------------------------------------------------------
-    // one accumulator per 16-column step (the instruction's latency is several hundred cycles: no step waits for
-    // another); the operand tiles are loaded four at a time
-    float acc[16][4];
+    // one accumulator per 16-column step (the steps do not wait for one another); the operand tiles are loaded
+    // four at a time
+    float acc[KS][4];
 #pragma unroll
-    for (int a = 0; a < 16; ++a)
+    for (int a = 0; a < KS; ++a)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][e] = 0.0f;
     {
       const unsigned char* src = (tile & 1) ? w_src : stage + x_off;
 #pragma unroll
-      for (int round = 0; round < 4; ++round) {
+      for (int round = 0; round < KS / 4; ++round) {
         uint32_t q[4][4];
 #pragma unroll
         for (int a = 0; a < 4; ++a)
@@ -425,7 +446,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
       }
     }
 #pragma unroll
-    for (int h = 8; h >= 1; h >>= 1)
+    for (int h = KS / 2; h >= 1; h >>= 1)
 #pragma unroll
       for (int a = 0; a < h; ++a)
 #pragma unroll
@@ -433,8 +454,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
     {
       // accumulator rows 0..7: lane l holds G[l / 4][2 (l % 4) .. +1]; rows 8..10 (lanes 0..11): the parts of p
       const int q = (int)(b & 1);
-      const uint32_t og = (uint32_t)__cvta_generic_to_shared(redG + ((size_t)q * MMA_SLOTS + slot) * MMA_G_VALS + lane * 2) - own_base;
-      const uint32_t op = (uint32_t)__cvta_generic_to_shared(redP + ((size_t)q * MMA_SLOTS + slot) * MMA_P_VALS + lane * 2) - own_base;
+      const uint32_t og = (uint32_t)__cvta_generic_to_shared(redG + ((size_t)q * SLOTS + slot) * MMA_G_VALS + lane * 2) - own_base;
+      const uint32_t op = (uint32_t)__cvta_generic_to_shared(redP + ((size_t)q * SLOTS + slot) * MMA_P_VALS + lane * 2) - own_base;
       const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&pbar[q]) - own_base;
 #pragma unroll
       for (int rr = 0; rr < 8; ++rr) {
@@ -445,10 +466,13 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
       }
     }
     // this thread's columns of the 8 rows, for the update: afterwards the stage can be refilled
-    uint4 raw[B];
+    uint32_t raw[B][NPL];
 #pragma unroll
-    for (int m = 0; m < B; ++m)
-      raw[m] = act ? *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16) : make_uint4(0u, 0u, 0u, 0u);
+    for (int m = 0; m < B; ++m) {
+#pragma unroll
+      for (int i = 0; i < NPL; ++i) raw[m][i] = 0u;
+      if (act) load_words(stage + (size_t)m * row_stride + (size_t)lc * LB, raw[m]);
+    }
     __syncthreads();  // gamma_b and the decision are in gam; every math warp is done with the stage
     if (gam[B + 1] != 0.0f) break;
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m, then the model rows again -----------------------------------------
@@ -462,10 +486,11 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
       const float ndl = -gam[B];
       const float2 ndl2 = make_float2(ndl, ndl);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < NPL; ++i) {
         float2 wv = __ffma2_rn(ndl2, w2[i], w2[i]);
 #pragma unroll
-        for (int m = 0; m < B; ++m) wv = __ffma2_rn(ngm2[m], XPairs<__nv_bfloat16>::get(raw[m], i), wv);
+        for (int m = 0; m < B; ++m)
+          wv = __ffma2_rn(ngm2[m], make_float2(__uint_as_float(raw[m][i] << 16), __uint_as_float(raw[m][i] & 0xffff0000u)), wv);
         w2[i] = wv;
       }
     }
@@ -475,10 +500,10 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma_kernel(const Cluster
   cluster_barrier();
 
   if (act) {
-    const long long c0 = (chunk0 + lc) * 8;
+    const long long c0 = chunk0 * 8 + (long long)lc * (2 * NPL);
     float* dst = p.W + (size_t)j * d + c0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NPL; ++i) {
       dst[2 * i] = w2[i].x;
       dst[2 * i + 1] = w2[i].y;
     }

@@ -70,6 +70,7 @@ struct wpsgd_ctx {
   long long opt_drop_block = -1;
   int opt_tc_gram = 0;
   int opt_chunks_per_thread = 0;  // cluster kernel: 16-byte chunks of a row per math thread (0: chosen here)
+  int opt_lane_bytes = 0;         // tensor-core cluster kernel: bytes of a row per math lane (0: chosen here, 8 or 16)
   int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
   int opt_timing = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -529,22 +530,27 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if (C != 1 && C != 2 && C != 4 && C != 8) return false;
   const long long cpc = (chunks + C - 1) / C;
   if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
-  const long long mw = (cpc + 31) / 32;
-  if (mw > 8 || mw * C > MMA_SLOTS) return false;
+  // bytes of a row per lane: 16 (one chunk, up to 8 math warps per CTA) unless asked otherwise (8: half a chunk, up
+  // to 16 math warps; measured slower on k = 128, d = 4096: 9.9 ms against 7.9 ms)
+  const int lane_bytes = c->opt_lane_bytes > 0 ? c->opt_lane_bytes : 16;
+  const int per_chunk = 16 / lane_bytes;
+  const long long mw = (cpc * per_chunk + 31) / 32;
+  const int slots = MMA_SLOTS * per_chunk;
+  if (mw > 8 * per_chunk || mw * C > slots) return false;
   // ring depth: as deep as asked for (default 2: a stage is free again as soon as its block has been through the
   // tensor-core pass, and a shallow ring lets more CTAs share an SM) while two CTAs still share an SM; else one per SM
   const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
   int want = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
   int stages = want;
-  while (stages > 2 && MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) --stages;
-  if (MmaSmem(stages, (size_t)cpc * 16).total > two_per_sm) {
+  while (stages > 2 && MmaSmem(stages, (size_t)cpc * 16, slots).total > two_per_sm) --stages;
+  if (MmaSmem(stages, (size_t)cpc * 16, slots).total > two_per_sm) {
     stages = want;
-    while (stages >= 2 && MmaSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
+    while (stages >= 2 && MmaSmem(stages, (size_t)cpc * 16, slots).total > kSmemBudget) --stages;
     if (stages < 2) return false;
   }
   out->C = C;
   out->cpc = (int)cpc;
-  out->R = 1;
+  out->R = per_chunk;  // lane units per 16-byte chunk
   out->math_warps = (int)mw;
   out->stages = stages;
   out->min_blocks = 2;
@@ -560,7 +566,7 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   cp.b.drop_block = c->opt_drop_block;
   cp.b.group_order = nullptr;
   cp.chunks_per_cta = sh.cpc;
-  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16).total;
+  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS * sh.R).total;
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
@@ -580,9 +586,9 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
     return WPSGD_OK;
   };
   switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_mma_kernel<LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_mma_kernel<LOSS_LOGISTIC>);
-    default: return go(chain_mma_kernel<LOSS_SQUARED>);
+    case WPSGD_LOSS_HINGE: return sh.R == 1 ? go(chain_mma_kernel<LOSS_HINGE, 4>) : go(chain_mma_kernel<LOSS_HINGE, 2>);
+    case WPSGD_LOSS_LOGISTIC: return sh.R == 1 ? go(chain_mma_kernel<LOSS_LOGISTIC, 4>) : go(chain_mma_kernel<LOSS_LOGISTIC, 2>);
+    default: return sh.R == 1 ? go(chain_mma_kernel<LOSS_SQUARED, 4>) : go(chain_mma_kernel<LOSS_SQUARED, 2>);
   }
 }
 
@@ -1044,6 +1050,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "cluster") {
     if (value < 0 || value > 16) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0..16");
     c->opt_cluster = (int)value;
+  } else if (n == "lane_bytes") {
+    if (value != 0 && value != 8 && value != 16) return fail(c, WPSGD_ERR_INVALID_ARG, "lane_bytes must be 0, 8 or 16");
+    c->opt_lane_bytes = (int)value;
   } else if (n == "chunks_per_thread") {
     if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "chunks_per_thread must be 0, 1 or 2");
     c->opt_chunks_per_thread = (int)value;

@@ -427,6 +427,18 @@ def test_mma_kernel_block_boundaries_and_ring_depths(P, n_steps, stages, variant
     assert_parity(P, wl, {"dense_variant": variant, "cluster": 2, "stages": stages})
 
 
+@pytest.mark.parametrize("d,cluster,loss", [(4096, 2, SQUARED), (488, 2, LOGISTIC), (264, 1, HINGE), (2048, 1, LOGISTIC), (1024, 8, SQUARED)])
+def test_mma_kernel_half_chunk_per_lane(P, d, cluster, loss):
+    # the narrower split (8 bytes of a row per lane, up to 16 math warps); the default is 16 bytes per lane
+    wl = wi.config2(k=4, d=d, m=48, base_steps=150)
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    wl.n_steps[1] = 7
+    wl.X = wl.X.to(torch.bfloat16)
+    assert_parity(P, wl, {"dense_variant": 8, "cluster": cluster, "lane_bytes": 8})
+
+
 @pytest.mark.parametrize("variant", TC_VARIANTS)
 def test_mma_kernel_model_split_keeps_fp32_accuracy(P, variant):
     # a model with a wide spread of magnitudes (w0 from 1e-6 to 1e3): the three bf16 rows must carry all 24 bits of
