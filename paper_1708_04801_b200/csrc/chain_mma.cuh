@@ -424,11 +424,12 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
     }
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
     // ---- [G_b ; p_b parts] over this warp's columns ------------------------------------------------------------
-    // one accumulator per 16-column step (the steps do not wait for one another); the operand tiles are loaded
-    // four at a time
-    float acc[KS][4];
+    // four independent accumulators (a dependent mma.sync takes about 20 cycles); the operand tiles are loaded four
+    // at a time
+    constexpr int NACC = 4;
+    float acc[NACC][4];
 #pragma unroll
-    for (int a = 0; a < KS; ++a)
+    for (int a = 0; a < NACC; ++a)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][e] = 0.0f;
     {
@@ -441,12 +442,11 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
           if (round * 4 + a < ksteps) ldmatrix_x4(q[a], src + (size_t)(round * 4 + a) * 32);
 #pragma unroll
         for (int a = 0; a < 4; ++a)
-          if (round * 4 + a < ksteps)
-            mma_bf16_m16n8k16(acc[round * 4 + a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
+          if (round * 4 + a < ksteps) mma_bf16_m16n8k16(acc[a], q[a][0], q[a][1], q[a][2], q[a][3], q[a][0], q[a][2]);
       }
     }
 #pragma unroll
-    for (int h = KS / 2; h >= 1; h >>= 1)
+    for (int h = NACC / 2; h >= 1; h >>= 1)
 #pragma unroll
       for (int a = 0; a < h; ++a)
 #pragma unroll
