@@ -36,7 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the chain kernel from an ncu capture, with the hash of the
 # kernel sources the capture was taken from; reported as null once the sources have changed.
-NCU_TRAFFIC = {"config2": {"src_sha": "5913da5afefb5bd9", "bytes_per_launch": 605861888}}
+NCU_TRAFFIC = {"config2": {"src_sha": "b0680cfd4ef4c937", "bytes_per_launch": 603605760}}
 
 
 def parse_args():
