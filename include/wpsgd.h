@@ -84,7 +84,8 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
  * picks for aligned bf16 rows of 2048 to 4096 columns); 9 bf16 rows, margins taken one block behind the model ("lagged" form);
  * 10 one CTA per node with the Gram block formed by warps of its own (rows of up to 256 16-byte chunks)), "cluster" (CTAs
  * per node of variants 7, 8, 9: 0 = chosen from d, else 1, 2, 4 or 8), "chunks_per_thread" (variant 7: 16-byte chunks of a
- * row per math thread, 0 = chosen, 1 or 2), "lane_bytes" (variant 8: bytes of a row per math lane, 0 = chosen, 8 or 16), "prefetch" (rows in
+ * row per math thread, 0 = chosen, 1 or 2), "lane_bytes" (variant 8: bytes of a row per math lane, 0 = chosen, 8 or 16), "host_pipeline" (wpsgd_solve_host: 1 (default) copies the shards in up to four
+ * groups of nodes, longest chains first, on a stream of the context and starts the chains of a group when its rows have arrived; 0 copies everything first), "prefetch" (rows in
  * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "stages" (blocks of 8 rows in the shared-memory ring of the blocked kernel; 0 = as many as fit, up to 4), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
  * (polls after which a device-side wait gives up), "tc_gram" (1: bf16 rows take the 8x8 Gram block of the blocked kernel from mma.sync tensor-core
  * instructions instead of FFMA; same result up to summation order), "test_drop_block" (test hook of the bounded wait: the rows of

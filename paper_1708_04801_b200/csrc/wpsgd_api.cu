@@ -73,6 +73,9 @@ struct wpsgd_ctx {
   int opt_lane_bytes = 0;         // tensor-core cluster kernel: bytes of a row per math lane (0: chosen here, 8 or 16)
   int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
   int opt_timing = 0;
+  int opt_host_pipeline = 1;  // host-buffer entry point: copy the shards in groups and start chains as they arrive
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_group[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   bool ev_valid = false;
   long long launches = 0;
@@ -883,8 +886,15 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   }
 }
 
+// Nodes launched together (a run of `count` consecutive entries of the longest-first order) once `ready` has happened.
+struct LaunchGroup {
+  int count;
+  cudaEvent_t ready;
+};
+
 wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long long ld, const float* y,
-                              const long long* shard_off, const long long* n_steps, const float* w0, bool resume) {
+                              const long long* shard_off, const long long* n_steps, const float* w0, bool resume,
+                              const std::vector<LaunchGroup>* groups = nullptr) {
   if (xt != WPSGD_X_F32 && xt != WPSGD_X_BF16) return fail(c, WPSGD_ERR_INVALID_ARG, "unknown feature type");
   if (ld < c->d) return fail(c, WPSGD_ERR_INVALID_ARG, "ld_elems < d");
   Plan pl;
@@ -903,8 +913,27 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
   p.status = c->status;
   s = timing_begin(c);
   if (s != WPSGD_OK) return s;
-  s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, p) : launch_dense<__nv_bfloat16>(c, p);
-  if (s != WPSGD_OK) return s;
+  if (!groups) {
+    s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, p) : launch_dense<__nv_bfloat16>(c, p);
+    if (s != WPSGD_OK) return s;
+  } else {
+    // one launch per group of nodes, each behind the event that says its rows are on the device
+    const int k_all = c->k;
+    int first_slot = 0;
+    for (const LaunchGroup& g : *groups) {
+      CU_TRY(c, cudaStreamWaitEvent(c->stream, g.ready, 0));
+      if (g.count > 0) {
+        ChainParams q = p;
+        q.order = c->t_order + first_slot;
+        q.k = g.count;
+        c->k = g.count;  // the launch helpers size their grids from it
+        s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, q) : launch_dense<__nv_bfloat16>(c, q);
+        c->k = k_all;
+        if (s != WPSGD_OK) return s;
+      }
+      first_slot += g.count;
+    }
+  }
   s = timing_end(c);
   if (s != WPSGD_OK) return s;
   for (int j = 0; j < c->k; ++j) c->steps_done[j] = first[j] + n_steps[j];
@@ -1027,6 +1056,10 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* c) {
     if (p) cudaFree(p);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  for (cudaEvent_t e : c->ev_group)
+    if (e) cudaEventDestroy(e);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   cudaGetLastError();
   delete c;
   return WPSGD_OK;
@@ -1050,6 +1083,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "cluster") {
     if (value < 0 || value > 16) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0..16");
     c->opt_cluster = (int)value;
+  } else if (n == "host_pipeline") {
+    if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "host_pipeline must be 0 or 1");
+    c->opt_host_pipeline = (int)value;
   } else if (n == "lane_bytes") {
     if (value != 0 && value != 8 && value != 16) return fail(c, WPSGD_ERR_INVALID_ARG, "lane_bytes must be 0, 8 or 16");
     c->opt_lane_bytes = (int)value;
@@ -1307,13 +1343,60 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, const
   if (s != WPSGD_OK) return s;
   if (!c->st_v) CU_TRY(c, cudaMalloc((void**)&c->st_v, (size_t)c->d * sizeof(float)));
   if (w0 && !c->st_w0) CU_TRY(c, cudaMalloc((void**)&c->st_w0, (size_t)c->d * sizeof(float)));
-  if (N > 0) {
-    CU_TRY(c, cudaMemcpyAsync(c->st_X, X, xbytes, cudaMemcpyHostToDevice, c->stream));
-    CU_TRY(c, cudaMemcpyAsync(c->st_y, y, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  // Pipelined form: the shards go to the device longest chain first on a copy stream of the context, in up to four
+  // groups of nodes, and the chains of a group start as soon as its rows have arrived, so all but the shortest chains
+  // run under the remaining copies. Not for rows of at most 64 chunks (their kernel packs nodes into CTAs over the
+  // whole node set) and not with fewer than two nodes.
+  const long long chunks = c->d / (long long)(16 / es);
+  const bool pipelined = c->opt_host_pipeline && N > 0 && c->k >= 2 && n_steps && chunks > 64;
+  if (!pipelined) {
+    if (N > 0) {
+      CU_TRY(c, cudaMemcpyAsync(c->st_X, X, xbytes, cudaMemcpyHostToDevice, c->stream));
+      CU_TRY(c, cudaMemcpyAsync(c->st_y, y, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    }
+    if (w0) CU_TRY(c, cudaMemcpyAsync(c->st_w0, w0, (size_t)c->d * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    s = wpsgd_run(c, c->st_X, xt, c->d, c->st_y, shard_off, n_steps, eta0, sched, lambda, loss, seed, w0 ? c->st_w0 : nullptr);
+    if (s != WPSGD_OK) return s;
+  } else {
+    s = check_hyper(c, eta0, (int)sched, lambda, (int)loss);
+    if (s != WPSGD_OK) return s;
+    for (int j = 0; j < c->k; ++j)
+      if (shard_off[j + 1] < shard_off[j] || shard_off[j] < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off is not non-decreasing");
+    if (!c->copy_stream) {
+      CU_TRY(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+      CU_TRY(c, cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+      for (cudaEvent_t& e : c->ev_group) CU_TRY(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    }
+    // the copies start after whatever the caller's stream still does with the staging buffers
+    CU_TRY(c, cudaEventRecord(c->ev_fork, c->stream));
+    CU_TRY(c, cudaStreamWaitEvent(c->copy_stream, c->ev_fork, 0));
+    CU_TRY(c, cudaMemcpyAsync(c->st_y, y, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+    if (w0) CU_TRY(c, cudaMemcpyAsync(c->st_w0, w0, (size_t)c->d * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+    std::vector<int> order(c->k);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return n_steps[a] > n_steps[b]; });  // as make_plan
+    const int n_groups = std::min(4, c->k);
+    std::vector<LaunchGroup> groups;
+    const size_t row_bytes = (size_t)c->d * es;
+    int slot = 0;
+    for (int g = 0; g < n_groups; ++g) {
+      const int count = (c->k - slot + (n_groups - g) - 1) / (n_groups - g);
+      for (int q = slot; q < slot + count; ++q) {
+        const int j = order[q];
+        const size_t off = (size_t)shard_off[j] * row_bytes, len = (size_t)(shard_off[j + 1] - shard_off[j]) * row_bytes;
+        if (len > 0)
+          CU_TRY(c, cudaMemcpyAsync((char*)c->st_X + off, (const char*)X + off, len, cudaMemcpyHostToDevice, c->copy_stream));
+      }
+      CU_TRY(c, cudaEventRecord(c->ev_group[g], c->copy_stream));
+      groups.push_back({count, c->ev_group[g]});
+      slot += count;
+    }
+    c->eta0 = eta0; c->sched = (int)sched; c->lambda = lambda; c->loss = (int)loss; c->seed = seed;
+    c->have_run = false;
+    s = run_dense_common(c, c->st_X, xt, c->d, c->st_y, (const long long*)shard_off, (const long long*)n_steps,
+                         w0 ? c->st_w0 : nullptr, false, &groups);
+    if (s != WPSGD_OK) return s;
   }
-  if (w0) CU_TRY(c, cudaMemcpyAsync(c->st_w0, w0, (size_t)c->d * sizeof(float), cudaMemcpyHostToDevice, c->stream));
-  s = wpsgd_run(c, c->st_X, xt, c->d, c->st_y, shard_off, n_steps, eta0, sched, lambda, loss, seed, w0 ? c->st_w0 : nullptr);
-  if (s != WPSGD_OK) return s;
   s = wpsgd_combine(c, r, c->st_v);
   if (s != WPSGD_OK) return s;
   CU_TRY(c, cudaMemcpyAsync(v_out, c->st_v, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));

@@ -749,6 +749,27 @@ def test_solve_host_equals_device_path(P):
     np.testing.assert_array_equal(again.numpy(), v_dev)
 
 
+@pytest.mark.parametrize("d,bf16,k", [(1024, False, 5), (1024, False, 2), (2048, True, 7), (480, False, 3)])
+@pytest.mark.parametrize("pipeline", [0, 1])
+def test_solve_host_pipelined_equals_device_path(P, d, bf16, k, pipeline):
+    # rows wide enough for the pipelined form: shards copied in groups (longest chains first), chains of a group
+    # launched when its rows have arrived; the per-node arithmetic is the same, so the result is bit for bit that of
+    # the device path
+    wl = wi.config2(k=k, d=d, m=96, base_steps=230)
+    wl.n_steps[k - 1] = 0
+    if bf16:
+        wl.X = wl.X.to(torch.bfloat16)
+    wl.w0 = torch.full((d,), 0.25)
+    v_dev, _, _, _ = gpu_solve(P, wl)
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("host_pipeline", pipeline)
+        for _ in range(2):
+            out = ctx.solve_host(wl.X.pin_memory(), wl.y.pin_memory(), wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam,
+                                 wl.loss, wl.seed, w0=wl.w0)
+            np.testing.assert_array_equal(out.numpy(), v_dev)
+        ctx.check()
+
+
 # ---- sparse path --------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
 @pytest.mark.parametrize("prefetch", [2, 4, 8])
