@@ -727,8 +727,12 @@ bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* s
   // (Measured on k = 1024, d = 256, speed ratio 4: 4.9 ms this way, 6.9 ms with one balanced 7-warp CTA per SM.)
   int warps = (int)std::min<long long>(4, std::max<long long>(1, c->k));
   if (c->opt_threads >= 32 && c->opt_threads % 32 == 0) warps = std::min(BLKW_MAX_WARPS, c->opt_threads / 32);
-  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 4) : 3;
-  while (BlockWarpSmem(stages, row_bytes, warps).total > (warps <= 4 ? 100 * 1024 : kSmemBudget)) {
+  // With at least four chains per SM in all, one CTA per SM (a ring of 4 stages per warp takes the shared memory of a
+  // second one) and the remaining CTAs queued behind, longest first, does a little better than two CTAs per SM
+  // (k = 1024: 4.76 ms against 4.98 ms): a warp alone on its scheduler takes about 2640 cycles per block, 3000 shared.
+  const bool one_cta_per_sm = c->opt_stages >= 4 || (c->opt_stages == 0 && c->k >= 4 * 148);
+  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 4) : (one_cta_per_sm ? 4 : 3);
+  while (BlockWarpSmem(stages, row_bytes, warps).total > ((warps <= 4 && !one_cta_per_sm) ? 100 * 1024 : kSmemBudget)) {
     if (stages > 2) --stages;
     else if (warps > 1) --warps;
     else return false;
