@@ -243,7 +243,7 @@ struct BlockSmem {
   }
 };
 
-template <typename XT, int R, int LOSS, bool OVERLAP, int MAXW, bool TC_GRAM>
+template <typename XT, int R, int LOSS, bool OVERLAP, int MAXW>
 __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;   // columns per 16-byte chunk
   constexpr int QV = V / 4;        // quads per chunk
@@ -257,10 +257,7 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
   const int j = p.order[blockIdx.x];
   const long long n_run = p.n_steps[j];
   const long long d = p.d;
-  // bf16 rows: the Gram block comes from the tensor cores (exact products, fp32 sums), which read 8x8 tiles
-  // across the 8 rows; 16 bytes of padding per staged row keep those reads free of bank conflicts
-  constexpr bool USE_MMA = TC_GRAM && (sizeof(XT) == 2);
-  constexpr int GW = USE_MMA ? 64 : 32;             // Gram partials per math warp
+  constexpr int GW = 32;  // Gram partials per math warp (28 used)
   const size_t row_bytes = (size_t)d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0);  // stride of a staged row
   const size_t ld_bytes = (size_t)p.ld * sizeof(XT);
   const BlockSmem L(S, row_bytes, math_warps);
@@ -339,24 +336,7 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       }
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       auto gather_gram = [&]() {
-        if (USE_MMA) {
-          // partials are full 8x8 blocks (row-major, symmetric); lane l sums entries l and l + 32
-          float g0[MAXW], g1[MAXW];
-#pragma unroll
-          for (int w = 0; w < MAXW; ++w) { g0[w] = redG[w * 64 + lane]; g1[w] = redG[w * 64 + 32 + lane]; }
-#pragma unroll
-          for (int h = MAXW / 2; h >= 1; h >>= 1)
-#pragma unroll
-            for (int w = 0; w < h; ++w) { g0[w] += g0[w + h]; g1[w] += g1[w + h]; }
-          totG[lane] = g0[0];
-          totG[32 + lane] = g1[0];
-          __syncwarp();
-#pragma unroll
-          for (int n2 = 1; n2 < B; ++n2)
-#pragma unroll
-            for (int m = 0; m < n2; ++m) Gs[n2 * (n2 - 1) / 2 + m] = totG[n2 * 8 + m] * sc[n2];
-          __syncwarp();
-        } else {
+        {
           float gp[MAXW];
 #pragma unroll
           for (int w = 0; w < MAXW; ++w) gp[w] = redG[w * 32 + lane];
@@ -591,31 +571,6 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
     const float ptot = warp_transpose_sum8(accp);
     if ((lane & 3) == 0) redP[mw * B + (lane >> 2)] = ptot;
   };
-  // Gram block of the rows in ring stage stg over this warp's columns, on the tensor cores: per 16 columns one
-  // m16n8k16 with A = the 8 rows (rows 8..15 of the tile zero) and B = the same rows as the "column" operand
-  auto gram_mma = [&](int stg) {
-    float gc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    const unsigned char* stage = ring + (size_t)stg * B * row_bytes;
-    const int row = lane & 7, mi = lane >> 3;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const long long seg0 = ((long long)r * TM + 32 * mw) * 8;  // first column of the warp's segment
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const long long col = seg0 + ks * 32;
-        if (col >= d) break;
-        const long long c = col + mi * 8;
-        uint32_t q[4];
-        ldmatrix_x4(q, stage + (size_t)row * row_bytes + (size_t)(c < d ? c : col) * 2);
-        if (col + 8 >= d) q[1] = 0u;
-        if (col + 16 >= d) q[2] = 0u;
-        if (col + 24 >= d) q[3] = 0u;
-        mma_bf16_m16n8k16(gc, q[0], 0u, q[1], 0u, q[0], q[1]);
-        mma_bf16_m16n8k16(gc, q[2], 0u, q[3], 0u, q[2], q[3]);
-      }
-    }
-    *(float2*)&redG[mw * 64 + (lane >> 2) * 8 + (lane & 3) * 2] = make_float2(gc[0], gc[1]);
-  };
   // w <- w - (1 - a^nv) w - sum_m gamma_m x_m with the rows held in raw
   auto update = [&](const uint4 (&raw)[R][B]) {
     float gm[B];
@@ -690,17 +645,11 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       load_raw(st, cur);
 #pragma unroll
       for (int m = 0; m < B; ++m) accp[m] = 0.0f;
-      if (USE_MMA) {
-        gram_mma(st);
-        products(cur, acc, accp, false, true);
-        publish_p(accp);
-      } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-        products(cur, acc, accp, true, true);
-        publish_p(accp);
-        publish_g(acc);
-      }
+      for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+      products(cur, acc, accp, true, true);
+      publish_p(accp);
+      publish_g(acc);
       __syncthreads();  // barrier 1: the stage of block b is free
       if (*give_up) break;
       __syncthreads();  // barrier 2: gamma_b is in gam

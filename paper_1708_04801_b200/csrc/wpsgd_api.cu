@@ -11,12 +11,8 @@
 #include <vector>
 
 #include "chain_block.cuh"
-#include "chain_cluster.cuh"
 #include "chain_csr.cuh"
-#include "chain_gram.cuh"
-#include "chain_lag.cuh"
 #include "chain_mma.cuh"
-#include "chain_tc.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
 #include "philox.cuh"
@@ -65,12 +61,9 @@ struct wpsgd_ctx {
   uint64_t seed = 0;
   // options
   int opt_stages = 0;
-  int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_block_rows = 0, opt_cluster = 0, opt_sparse_threads = 32;
+  int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_cluster = 0;
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
-  int opt_tc_gram = 0;
-  int opt_chunks_per_thread = 0;  // cluster kernel: 16-byte chunks of a row per math thread (0: chosen here)
-  int opt_lane_bytes = 0;         // tensor-core cluster kernel: bytes of a row per math lane (0: chosen here, 8 or 16)
   int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
   int opt_timing = 0;
   int opt_host_pipeline = 1;  // host-buffer entry point: copy the shards in groups and start chains as they arrive
@@ -284,10 +277,10 @@ wpsgd_status timing_end(wpsgd_ctx* c) {
 template <typename XT, int R, int PF>
 wpsgd_status launch_reg(wpsgd_ctx* c, const ChainParams& p, bool block_per_node, int threads) {
   if (block_per_node) {
-    chain_reg_kernel<XT, R, PF, true><<<c->k, threads, 0, c->stream>>>(p);
+    chain_reg_kernel<XT, R, PF, true><<<p.k, threads, 0, c->stream>>>(p);
   } else {
     const int nodes_per_cta = 4;
-    chain_reg_kernel<XT, R, PF, false><<<(c->k + nodes_per_cta - 1) / nodes_per_cta, 32 * nodes_per_cta, 0, c->stream>>>(p);
+    chain_reg_kernel<XT, R, PF, false><<<(p.k + nodes_per_cta - 1) / nodes_per_cta, 32 * nodes_per_cta, 0, c->stream>>>(p);
   }
   CU_TRY(c, cudaGetLastError());
   c->launches++;
@@ -330,11 +323,11 @@ bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* 
   return true;
 }
 
-template <typename XT, int R, bool OVL, int MAXW, bool TC>
+template <typename XT, int R, bool OVL, int MAXW>
 wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, size_t smem) {
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<c->k, threads, smem, c->stream>>>(bp);
+    kern<<<bp.c.k, threads, smem, c->stream>>>(bp);
     CU_TRY(c, cudaGetLastError());
     c->launches++;
     return WPSGD_OK;
@@ -342,9 +335,9 @@ wpsgd_status launch_block_r(wpsgd_ctx* c, const BlockParams& bp, int threads, si
   switch (c->loss) {
     // one 16-byte chunk per thread: room for two register copies of a block, so the Gram products of the
     // next block overlap the serial recurrence; more chunks: one copy, Gram and p in the same pass
-    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, OVL, MAXW, TC>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, OVL, MAXW, TC>);
-    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, OVL, MAXW, TC>);
+    case WPSGD_LOSS_HINGE: return go(chain_block_kernel<XT, R, LOSS_HINGE, OVL, MAXW>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_block_kernel<XT, R, LOSS_LOGISTIC, OVL, MAXW>);
+    default: return go(chain_block_kernel<XT, R, LOSS_SQUARED, OVL, MAXW>);
   }
 }
 
@@ -359,164 +352,21 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
   bp.group_order = nullptr;
   const size_t smem = BlockSmem(stages, (size_t)c->d * sizeof(XT) + (sizeof(XT) == 2 ? 16 : 0), threads / 32 - 2).total;
   const bool wide = threads > 64 + 32 * 8;  // more than 8 math warps: registers allow one copy of a block only
-  if (sizeof(XT) == 2) {
-    // bf16 rows: one register copy; the Gram block from FFMA (default) or from the tensor cores (option)
-    if (c->opt_tc_gram) {
-      if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, true>(c, bp, threads, smem)
-                              : launch_block_r<XT, 1, false, 8, true>(c, bp, threads, smem);
-      return wide ? launch_block_r<XT, 2, false, 16, true>(c, bp, threads, smem)
-                  : launch_block_r<XT, 2, false, 8, true>(c, bp, threads, smem);
-    }
-    if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, false>(c, bp, threads, smem)
-                            : launch_block_r<XT, 1, false, 8, false>(c, bp, threads, smem);
-    return wide ? launch_block_r<XT, 2, false, 16, false>(c, bp, threads, smem)
-                : launch_block_r<XT, 2, false, 8, false>(c, bp, threads, smem);
+  // one register copy of a block, except fp32 rows of at most 8 math warps with one chunk per thread (two copies:
+  // the Gram products of the next block overlap the recurrence)
+  if (R == 1) {
+    if (wide) return launch_block_r<XT, 1, false, 16>(c, bp, threads, smem);
+    return sizeof(XT) == 2 ? launch_block_r<XT, 1, false, 8>(c, bp, threads, smem)
+                           : launch_block_r<XT, 1, true, 8>(c, bp, threads, smem);
   }
-  if (R == 1) return wide ? launch_block_r<XT, 1, false, 16, false>(c, bp, threads, smem)
-                          : launch_block_r<XT, 1, true, 8, false>(c, bp, threads, smem);
-  return wide ? launch_block_r<XT, 2, false, 16, false>(c, bp, threads, smem)
-              : launch_block_r<XT, 2, false, 8, false>(c, bp, threads, smem);
-}
-
-// ---- blocked kernel with the Gram products on tcgen05 (bf16 rows) --------------------------------------------------
-bool tc_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out) {
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
-  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
-  if (c->d % 64 != 0) return false;
-  const long long chunks = c->d / 8;
-  const int R = (int)((chunks + 32 * TC_MATH_WARPS - 1) / (32 * TC_MATH_WARPS));
-  if (R > 2) return false;
-  const size_t row_bytes = (size_t)c->d * 2 + 16;
-  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 3;
-  while (stages >= 2 && TcSmem(stages, row_bytes).total > kSmemBudget) --stages;
-  if (stages < 2) return false;
-  *R_out = R;
-  *stages_out = stages;
-  return true;
-}
-
-template <int R>
-wpsgd_status launch_tc_r(wpsgd_ctx* c, const BlockParams& bp, size_t smem) {
-  auto go = [&](auto kern) -> wpsgd_status {
-    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<c->k, TC_THREADS, smem, c->stream>>>(bp);
-    CU_TRY(c, cudaGetLastError());
-    c->launches++;
-    return WPSGD_OK;
-  };
-  switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_tc_kernel<R, LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_tc_kernel<R, LOSS_LOGISTIC>);
-    default: return go(chain_tc_kernel<R, LOSS_SQUARED>);
-  }
-}
-
-wpsgd_status launch_tc(wpsgd_ctx* c, const ChainParams& p, int R, int stages) {
-  BlockParams bp;
-  bp.c = p;
-  bp.stages = stages;
-  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
-  bp.spin_limit = c->opt_spin_limit;
-  bp.drop_block = c->opt_drop_block;
-  bp.group_order = nullptr;
-  const size_t smem = TcSmem(stages, (size_t)c->d * 2 + 16).total;
-  return R == 1 ? launch_tc_r<1>(c, bp, smem) : launch_tc_r<2>(c, bp, smem);
-}
-
-// ---- blocked kernel with the columns of a chain split over a thread-block cluster -------------------------------
-struct ClusterShape {
-  int C = 1, cpc = 0, R = 1, math_warps = 1, stages = 2, min_blocks = 1;
-};
-
-// Shape of the cluster launch: C CTAs per chain (a power of two up to 8, the portable cluster size), cpc chunks of
-// a row per CTA, R chunks per math thread. Aim: about two CTAs per SM over the whole grid, so that the SMs of
-// finished chains keep working for the long ones, and at least one full warp of chunks per CTA.
-template <typename XT>
-bool cluster_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
-  constexpr int V = XVec<XT>::V;
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
-  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
-  const long long chunks = c->d / V;
-  if (chunks < 1) return false;
-  int C = c->opt_cluster;
-  if (C <= 0) {
-    C = 1;
-    while (C < 8 && (long long)c->k * (C * 2) <= 2 * 148 && chunks / (C * 2) >= 32) C *= 2;
-  }
-  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
-  const long long cpc = (chunks + C - 1) / C;
-  if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
-  int R = c->opt_chunks_per_thread;
-  if (R <= 0) R = cpc > 64 ? 2 : 1;
-  if (R != 1 && R != 2) return false;
-  const long long mw = (cpc + 32 * R - 1) / (32 * R);
-  if (mw > 8 || mw * C > CL_MAX_SLOTS) return false;
-  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
-  // two CTAs per SM when the ring allows it
-  const size_t per_cta_two = (size_t)(227 * 1024) / 2 - 1024;
-  int s2 = stages;
-  while (s2 >= 3 && ClusterSmem(s2, (size_t)cpc * 16).total > per_cta_two) --s2;
-  int min_blocks = 1;
-  if (s2 >= 3 && ClusterSmem(s2, (size_t)cpc * 16).total <= per_cta_two) {
-    stages = s2;
-    min_blocks = 2;
-  } else {
-    while (stages >= 2 && ClusterSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
-    if (stages < 2) return false;
-  }
-  out->C = C;
-  out->cpc = (int)cpc;
-  out->R = R;
-  out->math_warps = (int)mw;
-  out->stages = stages;
-  out->min_blocks = min_blocks;
-  return true;
-}
-
-template <typename XT, int R, int MAXMW, int MINB>
-wpsgd_status launch_cluster_r(wpsgd_ctx* c, const ClusterParams& cp, const ClusterShape& sh, size_t smem) {
-  auto go = [&](auto kern) -> wpsgd_status {
-    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
-    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = c->stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = (unsigned)sh.C;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = 1;
-    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
-    c->launches++;
-    return WPSGD_OK;
-  };
-  switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_cluster_kernel<XT, R, LOSS_HINGE, MAXMW, MINB>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_cluster_kernel<XT, R, LOSS_LOGISTIC, MAXMW, MINB>);
-    default: return go(chain_cluster_kernel<XT, R, LOSS_SQUARED, MAXMW, MINB>);
-  }
-}
-
-template <typename XT>
-wpsgd_status launch_cluster(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
-  ClusterParams cp;
-  cp.b.c = p;
-  cp.b.stages = sh.stages;
-  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
-  cp.b.spin_limit = c->opt_spin_limit;
-  cp.b.drop_block = c->opt_drop_block;
-  cp.b.group_order = nullptr;
-  cp.chunks_per_cta = sh.cpc;
-  const size_t smem = ClusterSmem(sh.stages, (size_t)sh.cpc * 16).total;
-  if (sh.R == 1) return launch_cluster_r<XT, 1, 8, 1>(c, cp, sh, smem);
-  if (sh.math_warps <= 4 && sh.min_blocks >= 2) return launch_cluster_r<XT, 2, 4, 2>(c, cp, sh, smem);
-  return launch_cluster_r<XT, 2, 8, 1>(c, cp, sh, smem);
+  return wide ? launch_block_r<XT, 2, false, 16>(c, bp, threads, smem) : launch_block_r<XT, 2, false, 8>(c, bp, threads, smem);
 }
 
 // ---- bf16 rows: Gram block and margins on the tensor cores, columns split over a cluster -------------------------------
+struct ClusterShape {
+  int C = 1, cpc = 0, math_warps = 1, stages = 2;
+};
+
 bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if (!aligned || c->sched != WPSGD_LR_CONST) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
@@ -533,13 +383,10 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   if (C != 1 && C != 2 && C != 4 && C != 8) return false;
   const long long cpc = (chunks + C - 1) / C;
   if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
-  // bytes of a row per lane: 16 (one chunk, up to 8 math warps per CTA) unless asked otherwise (8: half a chunk, up
-  // to 16 math warps; measured slower on k = 128, d = 4096: 9.9 ms against 7.9 ms)
-  const int lane_bytes = c->opt_lane_bytes > 0 ? c->opt_lane_bytes : 16;
-  const int per_chunk = 16 / lane_bytes;
-  const long long mw = (cpc * per_chunk + 31) / 32;
-  const int slots = MMA_SLOTS * per_chunk;
-  if (mw > 8 * per_chunk || mw * C > slots) return false;
+  // one 16-byte chunk of a row per lane, up to 8 math warps per CTA
+  const long long mw = (cpc + 31) / 32;
+  const int slots = MMA_SLOTS;
+  if (mw > 8 || mw * C > slots) return false;
   // ring depth: as deep as asked for (default 2: a stage is free again as soon as its block has been through the
   // tensor-core pass, and a shallow ring lets more CTAs share an SM) while two CTAs still share an SM; else one per SM
   const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
@@ -553,10 +400,8 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   }
   out->C = C;
   out->cpc = (int)cpc;
-  out->R = per_chunk;  // lane units per 16-byte chunk
   out->math_warps = (int)mw;
   out->stages = stages;
-  out->min_blocks = 2;
   return true;
 }
 
@@ -569,11 +414,11 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   cp.b.drop_block = c->opt_drop_block;
   cp.b.group_order = nullptr;
   cp.chunks_per_cta = sh.cpc;
-  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS * sh.R).total;
+  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
+    cfg.gridDim = dim3((unsigned)(p.k * sh.C));
     cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = c->stream;
@@ -589,131 +434,15 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
     return WPSGD_OK;
   };
   switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return sh.R == 1 ? go(chain_mma_kernel<LOSS_HINGE, 4>) : go(chain_mma_kernel<LOSS_HINGE, 2>);
-    case WPSGD_LOSS_LOGISTIC: return sh.R == 1 ? go(chain_mma_kernel<LOSS_LOGISTIC, 4>) : go(chain_mma_kernel<LOSS_LOGISTIC, 2>);
-    default: return sh.R == 1 ? go(chain_mma_kernel<LOSS_SQUARED, 4>) : go(chain_mma_kernel<LOSS_SQUARED, 2>);
-  }
-}
-
-// ---- bf16 rows: lagged blocked form (margins one block behind the model), columns split over a cluster -----------------------
-bool lag_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
-  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
-  const long long chunks = c->d / 8;
-  if (chunks < 1) return false;
-  int C = c->opt_cluster;
-  if (C <= 0) {
-    // a chain's speed is set by the tensor-core pass of its CTAs, so wide rows are split four ways; at least two full
-    // warps of chunks per CTA
-    C = 1;
-    while (C < 4 && chunks / (C * 2) >= 64) C *= 2;
-    while ((chunks + C - 1) / C > 256 && C < 8) C *= 2;  // a CTA takes at most 8 math warps of 32 chunks
-  }
-  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
-  const long long cpc = (chunks + C - 1) / C;
-  if ((long long)(C - 1) * cpc >= chunks) return false;  // every CTA of the cluster owns at least one chunk
-  const long long mw = (cpc + 31) / 32;
-  if (mw > 8 || mw * C > LAG_SLOTS) return false;
-  // ring depth (at least 3: the blocks i, i + 1 and i + 2 are in use at the same time): as deep as asked for
-  // (default 4) while two CTAs still share an SM; else one CTA per SM
-  const size_t two_per_sm = (size_t)(227 * 1024) / 2 - 1024;
-  int want = c->opt_stages > 0 ? std::min(std::max(c->opt_stages, 3), 8) : 4;
-  int stages = want;
-  while (stages > 3 && LagSmem(stages, (size_t)cpc * 16).total > two_per_sm) --stages;
-  if (LagSmem(stages, (size_t)cpc * 16).total > two_per_sm) {
-    stages = want;
-    while (stages >= 3 && LagSmem(stages, (size_t)cpc * 16).total > kSmemBudget) --stages;
-    if (stages < 3) return false;
-  }
-  out->C = C;
-  out->cpc = (int)cpc;
-  out->R = 1;
-  out->math_warps = (int)mw;
-  out->stages = stages;
-  out->min_blocks = 1;
-  return true;
-}
-
-wpsgd_status launch_lag(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
-  ClusterParams cp;
-  cp.b.c = p;
-  cp.b.stages = sh.stages;
-  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
-  cp.b.spin_limit = c->opt_spin_limit;
-  cp.b.drop_block = c->opt_drop_block;
-  cp.b.group_order = nullptr;
-  cp.chunks_per_cta = sh.cpc;
-  const size_t smem = LagSmem(sh.stages, (size_t)sh.cpc * 16).total;
-  auto go = [&](auto kern) -> wpsgd_status {
-    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->k * sh.C));
-    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = c->stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = (unsigned)sh.C;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = 1;
-    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
-    c->launches++;
-    return WPSGD_OK;
-  };
-  switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_lag_kernel<LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_lag_kernel<LOSS_LOGISTIC>);
-    default: return go(chain_lag_kernel<LOSS_SQUARED>);
-  }
-}
-
-// ---- blocked kernel with Gram warps (one CTA per node, rows of up to 256 chunks) ---------------------------------------
-template <typename XT>
-bool gram_kernel_fits(const wpsgd_ctx* c, bool aligned, int* math_warps_out, int* stages_out) {
-  constexpr int V = XVec<XT>::V;
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
-  if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
-  const long long chunks = c->d / V;
-  if (chunks < 1 || chunks > 32 * GRAM_MAX_MATH_WARPS) return false;
-  const size_t row_bytes = (size_t)c->d * sizeof(XT);
-  int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 4;
-  while (stages >= 2 && GramSmem(stages, row_bytes).total > kSmemBudget) --stages;
-  if (stages < 2) return false;
-  *math_warps_out = (int)((chunks + 31) / 32);
-  *stages_out = stages;
-  return true;
-}
-
-template <typename XT>
-wpsgd_status launch_gram(wpsgd_ctx* c, const ChainParams& p, int math_warps, int stages) {
-  BlockParams bp;
-  bp.c = p;
-  bp.stages = stages;
-  bp.eta_lambda = (double)c->eta0 * (double)c->lambda;
-  bp.spin_limit = c->opt_spin_limit;
-  bp.drop_block = c->opt_drop_block;
-  bp.group_order = nullptr;
-  const size_t smem = GramSmem(stages, (size_t)c->d * sizeof(XT)).total;
-  const int threads = 64 + 32 * math_warps + 32 * ((math_warps + 1) / 2);  // math warps and one Gram warp per 64 chunks
-  auto go = [&](auto kern) -> wpsgd_status {
-    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<c->k, threads, smem, c->stream>>>(bp);
-    CU_TRY(c, cudaGetLastError());
-    c->launches++;
-    return WPSGD_OK;
-  };
-  switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_gram_kernel<XT, LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_gram_kernel<XT, LOSS_LOGISTIC>);
-    default: return go(chain_gram_kernel<XT, LOSS_SQUARED>);
+    case WPSGD_LOSS_HINGE: return go(chain_mma_kernel<LOSS_HINGE, 4>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_mma_kernel<LOSS_LOGISTIC, 4>);
+    default: return go(chain_mma_kernel<LOSS_SQUARED, 4>);
   }
 }
 
 // blocked kernel, one warp per node (small d)
 template <typename XT>
-bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* stages_out, int* warps_out) {
+bool block_warp_kernel_fits(const wpsgd_ctx* c, int nk, bool aligned, int* R_out, int* stages_out, int* warps_out) {
   constexpr int V = XVec<XT>::V;
   if (!aligned || c->sched != WPSGD_LR_CONST) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
@@ -725,12 +454,13 @@ bool block_warp_kernel_fits(const wpsgd_ctx* c, bool aligned, int* R_out, int* s
   // a long chain needs is few co-runners late in the run, not an equal share of work per SM: with chains dealt out
   // longest first, the CTAs of the longest chains land on the SMs first and are paired with the shortest ones.
   // (Measured on k = 1024, d = 256, speed ratio 4: 4.9 ms this way, 6.9 ms with one balanced 7-warp CTA per SM.)
-  int warps = (int)std::min<long long>(4, std::max<long long>(1, c->k));
+  if (nk != c->k) return false;  // its node-to-CTA table covers the whole node set
+  int warps = (int)std::min<long long>(4, std::max<long long>(1, nk));
   if (c->opt_threads >= 32 && c->opt_threads % 32 == 0) warps = std::min(BLKW_MAX_WARPS, c->opt_threads / 32);
   // With at least four chains per SM in all, one CTA per SM (a ring of 4 stages per warp takes the shared memory of a
   // second one) and the remaining CTAs queued behind, longest first, does a little better than two CTAs per SM
   // (k = 1024: 4.76 ms against 4.98 ms): a warp alone on its scheduler takes about 2640 cycles per block, 3000 shared.
-  const bool one_cta_per_sm = c->opt_stages >= 4 || (c->opt_stages == 0 && c->k >= 4 * 148);
+  const bool one_cta_per_sm = c->opt_stages >= 4 || (c->opt_stages == 0 && nk >= 4 * 148);
   int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 4) : (one_cta_per_sm ? 4 : 3);
   while (BlockWarpSmem(stages, row_bytes, warps).total > ((warps <= 4 && !one_cta_per_sm) ? 100 * 1024 : kSmemBudget)) {
     if (stages > 2) --stages;
@@ -798,7 +528,7 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   int bthreads = 0, bR = 0, bstages = 0;
   const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
   int wR = 0, wstages = 0, wwarps = 0;
-  const bool block_warp_ok = block_warp_kernel_fits<XT>(c, aligned, &wR, &wstages, &wwarps);
+  const bool block_warp_ok = block_warp_kernel_fits<XT>(c, p.k, aligned, &wR, &wstages, &wwarps);
   ClusterShape mma_shape;
   const bool mma_ok = sizeof(XT) == 2 && mma_kernel_fits(c, aligned, &mma_shape);
   if (variant == 0) {
@@ -815,21 +545,6 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
   }
-  if (variant == 10) {
-    int gmw = 0, gstages = 0;
-    if (!gram_kernel_fits<XT>(c, aligned, &gmw, &gstages))
-      return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "Gram-warp kernel needs 16-byte aligned rows of at most 256 chunks, a constant step size and eta*lambda <= 0.25");
-    return launch_gram<XT>(c, p, gmw, gstages);
-  }
-  if (variant == 9) {
-    ClusterShape sh;
-    if (sizeof(XT) != 2 || !lag_kernel_fits(c, aligned, &sh))
-      return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "lagged cluster kernel needs bf16 rows, 16-byte aligned, a constant step size, eta*lambda <= 0.25, a "
-                  "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
-    return launch_lag(c, p, sh);
-  }
   if (variant == 8) {
     ClusterShape sh;
     if (sizeof(XT) != 2 || !mma_kernel_fits(c, aligned, &sh))
@@ -837,22 +552,6 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "tensor-core cluster kernel needs bf16 rows, 16-byte aligned, a constant step size, eta*lambda <= 0.25, a "
                   "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
     return launch_mma(c, p, sh);
-  }
-  if (variant == 7) {
-    ClusterShape sh;
-    if (!cluster_kernel_fits<XT>(c, aligned, &sh))
-      return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "cluster kernel needs 16-byte aligned rows, a constant step size, eta*lambda <= 0.25, a cluster of 1, 2, 4 "
-                  "or 8 CTAs with at most 512 chunks of a row each and at most 16 math warps in all");
-    return launch_cluster<XT>(c, p, sh);
-  }
-  if (variant == 6 || (variant == 4 && c->opt_tc_gram == 2)) {
-    int tR = 0, tstages = 0;
-    if (sizeof(XT) != 2 || !tc_kernel_fits(c, aligned, &tR, &tstages))
-      return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "tcgen05 kernel needs bf16 rows, 16-byte aligned, d a multiple of 64 and at most 4096, a constant "
-                  "step size and eta*lambda <= 0.25");
-    return launch_tc(c, p, tR, tstages);
   }
   if (variant == 4) {
     if (!block_ok)
@@ -865,7 +564,7 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   if (variant == 3 && chunks > 32 * 4) return fail(c, WPSGD_ERR_UNSUPPORTED, "warp-per-node kernel: d too large");
   if (variant == 2 && chunks > 512 * 4) return fail(c, WPSGD_ERR_UNSUPPORTED, "CTA-per-node kernel: d too large");
   if (variant == 1) {
-    chain_generic_kernel<XT><<<c->k, 256, 0, c->stream>>>(p);
+    chain_generic_kernel<XT><<<p.k, 256, 0, c->stream>>>(p);
     CU_TRY(c, cudaGetLastError());
     c->launches++;
     return WPSGD_OK;
@@ -922,7 +621,6 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
     if (s != WPSGD_OK) return s;
   } else {
     // one launch per group of nodes, each behind the event that says its rows are on the device
-    const int k_all = c->k;
     int first_slot = 0;
     for (const LaunchGroup& g : *groups) {
       CU_TRY(c, cudaStreamWaitEvent(c->stream, g.ready, 0));
@@ -930,9 +628,7 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
         ChainParams q = p;
         q.order = c->t_order + first_slot;
         q.k = g.count;
-        c->k = g.count;  // the launch helpers size their grids from it
-        s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, q) : launch_dense<__nv_bfloat16>(c, q);
-        c->k = k_all;
+        s = (xt == WPSGD_X_F32) ? launch_dense<float>(c, q) : launch_dense<__nv_bfloat16>(c, q);  // grids follow q.k
         if (s != WPSGD_OK) return s;
       }
       first_slot += g.count;
@@ -1073,7 +769,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 10) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..10");
+    if (value < 0 || value > 8 || value == 6 || value == 7) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..5 or 8");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");
@@ -1081,24 +777,12 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "threads") {
     if (value != 0 && (value < 32 || value > 512 || value % 32)) return fail(c, WPSGD_ERR_INVALID_ARG, "threads must be 0 or a multiple of 32 in 32..512");
     c->opt_threads = (int)value;
-  } else if (n == "block_rows") {
-    if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "block_rows must be 0..64");
-    c->opt_block_rows = (int)value;
   } else if (n == "cluster") {
-    if (value < 0 || value > 16) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0..16");
+    if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return fail(c, WPSGD_ERR_INVALID_ARG, "cluster must be 0, 1, 2, 4 or 8");
     c->opt_cluster = (int)value;
   } else if (n == "host_pipeline") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "host_pipeline must be 0 or 1");
     c->opt_host_pipeline = (int)value;
-  } else if (n == "lane_bytes") {
-    if (value != 0 && value != 8 && value != 16) return fail(c, WPSGD_ERR_INVALID_ARG, "lane_bytes must be 0, 8 or 16");
-    c->opt_lane_bytes = (int)value;
-  } else if (n == "chunks_per_thread") {
-    if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "chunks_per_thread must be 0, 1 or 2");
-    c->opt_chunks_per_thread = (int)value;
-  } else if (n == "sparse_threads") {
-    if (value != 32) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_threads must be 32");
-    c->opt_sparse_threads = (int)value;
   } else if (n == "stages") {
     if (value < 0 || value == 1 || value > 8) return fail(c, WPSGD_ERR_INVALID_ARG, "stages must be 0 or 2..8");
     c->opt_stages = (int)value;
@@ -1108,9 +792,6 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "sampling") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "sampling must be 0 (i.i.d. draws) or 1 (shuffled order)");
     c->opt_sampling = (int)value;
-  } else if (n == "tc_gram") {
-    if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "tc_gram must be 0, 1 or 2");
-    c->opt_tc_gram = (int)value;
   } else if (n == "test_drop_block") {
     c->opt_drop_block = value;
   } else if (n == "spin_limit") {
