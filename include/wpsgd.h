@@ -70,27 +70,37 @@ wpsgd_status wpsgd_create(int device, void* cuda_stream, int32_t k, int64_t d, w
 /* Release everything the context owns. Synchronises the stream first. NULL is accepted. */
 wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
 
-/* Options by name. "sampling": order of the examples. 0 (default) = independent uniform draws as described in the
- * header comment. 1 = the literal reading of Algorithm 1 ("randomly shuffle the data on machine i", then "get the
- * n-th example"): one fixed pseudo-random permutation pi_j of the shard per node, cycled, i.e. the n-th example
- * is row pi_j((n-1) mod m_j); pi_j is a 4-round balanced Feistel network on the even bit count covering m_j - 1
- * with cycle walking, keyed by the Philox block at counter (0, 0, j, 1) under the seed, round function
- * mix(R ^ key) = multiply 0x85EBCA6B, xor-shift 13, multiply 0xC2B2AE35, xor-shift 16, masked to half the bits.
- * Kernel selection and tuning, by name. Names: "dense_variant" (0 auto, 1 generic, 2 CTA per node
- * with register-held model, 3 warp per node, 4 blocked kernel: 8 samples per synchronisation, CTA per node; 5 the same with a warp per node; 6 the blocked kernel for bf16 rows with the Gram products on
- * tcgen05 tensor cores, 64 samples at a time (kept for comparison: measured slower than 4 on B200); 7 the blocked form with the
- * columns of a node split over a thread-block cluster, packed fp32 FMAs; 8 the same split for bf16 rows with the Gram block
- * and the margins of a block from mma.sync tensor-core instructions, the fp32 model entering as three bf16 rows (what 0
- * picks for aligned bf16 rows of 2048 to 4096 columns); 9 bf16 rows, margins taken one block behind the model ("lagged" form);
- * 10 one CTA per node with the Gram block formed by warps of its own (rows of up to 256 16-byte chunks)), "cluster" (CTAs
- * per node of variants 7, 8, 9: 0 = chosen from d, else 1, 2, 4 or 8), "chunks_per_thread" (variant 7: 16-byte chunks of a
- * row per math thread, 0 = chosen, 1 or 2), "lane_bytes" (variant 8: bytes of a row per math lane, 0 = chosen, 8 or 16), "host_pipeline" (wpsgd_solve_host: 1 (default) copies the shards in up to four
- * groups of nodes, longest chains first, on a stream of the context and starts the chains of a group when its rows have arrived; 0 copies everything first), "prefetch" (rows in
- * flight per chain), "threads" (threads per node of variant 2; 0 = chosen from d), "stages" (blocks of 8 rows in the shared-memory ring of the blocked kernel; 0 = as many as fit, up to 4), "sparse_threads" (threads per node of the CSR kernel), "spin_limit"
- * (polls after which a device-side wait gives up), "tc_gram" (1: bf16 rows take the 8x8 Gram block of the blocked kernel from mma.sync tensor-core
- * instructions instead of FFMA; same result up to summation order), "test_drop_block" (test hook of the bounded wait: the rows of
- * that block of every chain are never requested, so the wait for them runs out; -1 = off), "timing" (1: record events around the chain kernel). Unknown name or bad value:
- * WPSGD_ERR_INVALID_ARG. The result of a run never depends on these beyond rounding order. */
+/* Options by name. Unknown name or bad value: WPSGD_ERR_INVALID_ARG. Except for "sampling", the result of a run
+ * never depends on an option beyond rounding order.
+ *
+ *   "sampling"        order of the examples. 0 (default): independent uniform draws as in the header comment.
+ *                     1: the literal reading of Algorithm 1 ("randomly shuffle the data on machine i", then "get the
+ *                     n-th example"): one fixed pseudo-random permutation pi_j of the shard per node, cycled, i.e. the
+ *                     n-th example is row pi_j((n-1) mod m_j). pi_j is a 4-round balanced Feistel network on the even
+ *                     bit count covering m_j - 1 with cycle walking, keyed by the Philox block at counter (0, 0, j, 1)
+ *                     under the seed; round function mix(R ^ key) = multiply 0x85EBCA6B, xor-shift 13, multiply
+ *                     0xC2B2AE35, xor-shift 16, masked to half the bits.
+ *   "dense_variant"   kernel for dense rows. 0 (default): chosen from the shape. 1: any shape and alignment, model in
+ *                     global memory. 2: one CTA per node, one step per round trip, model in registers. 3: the same with
+ *                     one warp per node. 4: blocked form (8 samples per synchronisation), one CTA per node. 5: blocked
+ *                     form, one warp per node (rows of at most 64 16-byte chunks). 8: blocked form for bf16 rows, Gram
+ *                     block and margins from mma.sync tensor-core instructions, columns of a node split over a
+ *                     thread-block cluster (what 0 picks for aligned bf16 rows of 2048 columns and more).
+ *   "sparse_variant"  kernel for CSR rows. 0 (default) and 2: blocks of up to 64 steps run in a shared-memory cache of
+ *                     the model entries they touch. 1: one step per round trip to the model in global memory.
+ *   "cluster"         CTAs per node of variant 8: 0 (default) chosen from d, else 1, 2, 4 or 8.
+ *   "threads"         threads per node of variants 2 and 4, warps x 32 per CTA of variant 5; 0 (default): chosen from d.
+ *   "prefetch"        rows in flight per chain of variants 2, 3 and of sparse variant 1; 0 (default): chosen.
+ *   "stages"          blocks of rows in the shared-memory ring of the blocked kernels; 0 (default): as many as fit
+ *                     (up to 4), else 2..8.
+ *   "host_pipeline"   wpsgd_solve_host: 1 (default) copies the shards in up to four groups of nodes, longest chains
+ *                     first, on a stream of the context and starts the chains of a group when its rows have arrived;
+ *                     0 copies everything first.
+ *   "spin_limit"      polls after which a device-side wait gives up (default 2^20).
+ *   "timing"          1: record events around the chain kernel (see wpsgd_last_chain_ms). Default 0.
+ *   "test_drop_block" test hook of the bounded waits, not for production use: the rows of that block of every chain
+ *                     are never requested, so the wait for them runs out and WPSGD_ERR_TIMEOUT is reported by
+ *                     wpsgd_check; -1 (default) = off. */
 wpsgd_status wpsgd_set_option(wpsgd_ctx* ctx, const char* name, int64_t value);
 
 /* Node numbers that enter the sample stream in place of 0..k-1 (HOST [k], >= 0; NULL restores the
@@ -117,7 +127,8 @@ wpsgd_status wpsgd_run(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld
  * numbered after the ones it has already run (so it draws examples step_done+1, ...). Data and
  * hyper-parameters must be the ones given to the wpsgd_run / wpsgd_run_csr that started the
  * chains. Gives the paper's snapshots "after 100000 x i updates of the fastest node"
- * (Section "Numerical experiments", Approach) without restarting. Dense data only. */
+ * (Section "Numerical experiments", Approach) without restarting. Dense rows; chains that were started on CSR
+ * rows continue with wpsgd_continue_csr. */
 wpsgd_status wpsgd_continue(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64_t ld_elems, const float* y,
                             const int64_t* shard_off, const int64_t* n_more);
 
@@ -129,6 +140,20 @@ wpsgd_status wpsgd_continue(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, int64
 wpsgd_status wpsgd_run_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
                            const float* y, const int64_t* shard_off, const int64_t* n_steps, float eta0,
                            wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed, const float* w0);
+
+/* wpsgd_continue on CSR rows: node j runs n_more[j] further steps from the model (u_j and its scale) the context
+ * holds; arrays as wpsgd_run_csr, hyper-parameters and seed those of the run that started the chains. With
+ * wpsgd_combine and wpsgd_set_models this is averaging every `span` fastest-node steps on the paper's kind of data
+ * (Section "Combining WP-SGD with bucket SGD"). */
+wpsgd_status wpsgd_continue_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                                const float* y, const int64_t* shard_off, const int64_t* n_more);
+
+/* Read-only check of a CSR matrix against the preconditions of wpsgd_run_csr, enqueued on the context's stream:
+ * row_ptr DEVICE [n_rows+1] within [0, nnz] and non-decreasing, col_idx DEVICE [nnz] in [0, d) and strictly increasing
+ * within a row (no column twice: the sparse update of Eq. 5 writes each nonzero's model entry once). Nothing outside
+ * [0, nnz) is read. A violation is reported by the next wpsgd_check as WPSGD_ERR_CUDA with the row in the message. */
+wpsgd_status wpsgd_validate_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, int64_t n_rows,
+                                int64_t nnz);
 
 /* Algorithm 1, the aggregation: v = sum_j weight_j w_j (j ascending) with Eq. 6 weights, or Eq. 8
  * weights when r > 0 is given (r <= 0 or NaN selects the default; r = 1 is plain averaging).
@@ -158,6 +183,20 @@ wpsgd_status wpsgd_get_weights(wpsgd_ctx* ctx, double r, double* weights, int* c
  * sum_j r^{T_j}, the quantity in Eq. 7 / Eq. 9 and in the validity bound of averaging every span. */
 wpsgd_status wpsgd_weights(const int64_t* n_steps, int32_t k, float eta0, wpsgd_lr sched, float lambda,
                            double r, double* weights, int* cond_holds, double* sum_rT);
+
+/* Condition the paper gives for averaging every `span` fastest-node steps on an unbalanced system (Section "Combining
+ * WP-SGD with bucket SGD", after Deduction 2): (k / sum_j r^{T_j}) (1 - eta lambda)^span < 1, with r = 1 - eta lambda
+ * unless r > 0 is given. n_steps HOST [k]. lhs (may be NULL) receives the left-hand side, holds (may be NULL) whether
+ * it is below 1. Constant step size. Host-only computation. */
+wpsgd_status wpsgd_span_valid(const int64_t* n_steps, int32_t k, float eta0, float lambda, double r, int64_t span,
+                              double* lhs, int* holds);
+
+/* The sample stream of Algorithm 1's "get the n-th example" as defined in the header comment, computed on the host by
+ * the same function the kernels call: row indices (within a shard of m rows) of steps n_begin+1 .. n_begin+count of
+ * node `node`, to out HOST [count] uint32. sampling as the option of that name (0 draws, 1 shuffled order). Needs no
+ * context and no GPU. */
+wpsgd_status wpsgd_sample_indices_host(uint64_t seed, int32_t node, int64_t m, int64_t n_begin, int64_t count,
+                                       int32_t sampling, uint32_t* out);
 
 /* The sample stream exactly as the chain kernels draw it: row indices (within the shard of m rows)
  * of steps n_begin+1 .. n_begin+count of node `node`, to out DEVICE [count] uint32. */
@@ -189,7 +228,7 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, con
  * this is a convenience of the library.) It does what wpsgd_run followed by wpsgd_combine does on
  * dense rows, but takes no context and calls no cudaMalloc / cudaFree or any other allocating
  * routine: the model matrix, the sample stream and the small tables that a context would own live in
- * one array built into the library (about 5.1 MiB of device memory on every GPU that loads it, held
+ * one array built into the library (about 5.4 MiB of device memory on every GPU that loads it, held
  * until the process exits). Meant for code that runs where allocation is forbidden or would stall:
  * inside another framework's memory pool that has reserved the whole device, in a latency-critical
  * loop that cannot afford cudaMalloc's device-wide synchronisation, or in a process whose memory
@@ -204,7 +243,9 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, con
  * first call before starting any stream capture. All calls on a device share the one array, which
  * still holds what the previous call left there; each call rewrites what it uses and clears its
  * status word, so calls in sequence on one stream are independent, but two calls whose GPU work
- * overlaps (different streams, or different host threads) race on it and give wrong results. */
+ * overlaps (different streams, or different host threads) race on it and give wrong results.
+ * The kernels' status word (a bounded wait that gave up, a failed bounds check) lives in the same array;
+ * wpsgd_check_static reads it. */
 #define WPSGD_STATIC_MAX_NODES 1024
 #define WPSGD_STATIC_MAX_MODEL_ELEMS (1 << 18)
 #define WPSGD_STATIC_MAX_STEPS (1 << 20)
@@ -212,6 +253,10 @@ wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wp
                                 const float* y, const int64_t* shard_off, const int64_t* n_steps, int32_t k,
                                 int64_t d, float eta0, wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed,
                                 const float* w0, double r, float* v_out);
+
+/* wpsgd_check for wpsgd_solve_static: waits for the stream and reads the status word inside the built-in array
+ * (no allocation). Same return values as wpsgd_check; the text is available from wpsgd_last_error(NULL). */
+wpsgd_status wpsgd_check_static(int device, void* cuda_stream);
 
 /* Wait for the stream and read the device status word. WPSGD_OK, WPSGD_ERR_TIMEOUT (a bounded wait
  * gave up), or WPSGD_ERR_CUDA (a launch or copy failed, or a kernel's own bounds check fired). */

@@ -7,5 +7,5 @@ build step itself can import the package), but any call raises if it is missing.
 """
 from .binding import (  # noqa: F401
     LOSS_HINGE, LOSS_LOGISTIC, LOSS_SQUARED, LR_CONST, LR_INV_SQRT, X_BF16, X_F32, WpsgdError, Context,
-    library_path, load_library, weights, solve_static, averaging_span_valid, EXPORTED_SYMBOLS,
+    library_path, load_library, weights, solve_static, span_valid, sample_indices_host, check_static, EXPORTED_SYMBOLS,
 )

@@ -17,7 +17,8 @@ EXPORTED_SYMBOLS = [
     "wpsgd_create", "wpsgd_destroy", "wpsgd_set_option", "wpsgd_set_node_ids", "wpsgd_run", "wpsgd_continue", "wpsgd_run_csr",
     "wpsgd_combine", "wpsgd_combine_weighted", "wpsgd_last_chain_ms", "wpsgd_get_models", "wpsgd_set_models", "wpsgd_get_weights", "wpsgd_weights",
     "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_objective_csr", "wpsgd_solve_host", "wpsgd_solve_static", "wpsgd_check", "wpsgd_launch_count",
-    "wpsgd_last_error",
+    "wpsgd_last_error", "wpsgd_continue_csr", "wpsgd_validate_csr", "wpsgd_span_valid", "wpsgd_sample_indices_host",
+    "wpsgd_check_static",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -68,6 +69,11 @@ def load_library() -> ctypes.CDLL:
     lib.wpsgd_solve_host.argtypes = [vp, vp, ci, vp, vp, vp, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_solve_static.argtypes = [ci, vp, vp, ci, i64, vp, vp, vp, i32, i64, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_check.argtypes = [vp]
+    lib.wpsgd_continue_csr.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.wpsgd_validate_csr.argtypes = [vp, vp, vp, i64, i64]
+    lib.wpsgd_span_valid.argtypes = [vp, i32, f32, f32, f64, i64, ctypes.POINTER(f64), ctypes.POINTER(ci)]
+    lib.wpsgd_sample_indices_host.argtypes = [u64, i32, i64, i64, i64, i32, vp]
+    lib.wpsgd_check_static.argtypes = [ci, vp]
     lib.wpsgd_launch_count.argtypes = [vp]
     lib.wpsgd_launch_count.restype = i64
     lib.wpsgd_last_error.argtypes = [vp]
@@ -97,14 +103,39 @@ def weights(n_steps, eta0: float, sched: int, lam: float, r: float = 0.0) -> Tup
     return w, bool(flag.value), float(tot.value)
 
 
-def averaging_span_valid(n_steps, eta0: float, lam: float, span: int, r: float = 0.0) -> Tuple[bool, float]:
-    """Condition the paper gives for averaging every `span` fastest-node steps on an unbalanced system
-    (Section "Combining WP-SGD with bucket SGD"): (k / sum_j r^{T_j}) * (1 - eta lambda)^span < 1.
-    Returns (holds, left-hand side); sum_j r^{T_j} comes from wpsgd_weights."""
+def span_valid(n_steps, eta0: float, lam: float, span: int, r: float = 0.0) -> Tuple[bool, float]:
+    """wpsgd_span_valid: the paper's condition for averaging every `span` fastest-node steps on an unbalanced
+    system, (k / sum_j r^{T_j}) (1 - eta lambda)^span < 1. Returns (holds, left-hand side)."""
+    lib = load_library()
     n = _host_i64(n_steps)
-    _, _, tot = weights(n, eta0, LR_CONST, lam, r)
-    lhs = (n.shape[0] / tot) * (1.0 - float(np.float32(eta0)) * float(np.float32(lam))) ** int(span)
-    return bool(lhs < 1.0), float(lhs)
+    lhs = ctypes.c_double(0.0)
+    flag = ctypes.c_int(0)
+    st = lib.wpsgd_span_valid(n.ctypes.data, n.shape[0], eta0, lam, r, int(span), ctypes.byref(lhs), ctypes.byref(flag))
+    if st:
+        raise WpsgdError(st, "wpsgd_span_valid", lib.wpsgd_last_error(None).decode())
+    return bool(flag.value), float(lhs.value)
+
+
+def sample_indices_host(seed: int, node: int, m: int, n_begin: int, count: int, sampling: int = 0) -> np.ndarray:
+    """wpsgd_sample_indices_host: the sample stream of the chains, computed on the host by the library."""
+    lib = load_library()
+    out = np.zeros(max(count, 0), dtype=np.uint32)
+    st = lib.wpsgd_sample_indices_host(seed, node, m, n_begin, count, sampling, out.ctypes.data if count > 0 else None)
+    if st:
+        raise WpsgdError(st, "wpsgd_sample_indices_host", lib.wpsgd_last_error(None).decode())
+    return out
+
+
+def check_static(device: int = 0, stream=None):
+    """wpsgd_check_static: wait for the stream and read the status word of wpsgd_solve_static's built-in array."""
+    import torch
+
+    lib = load_library()
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    st = lib.wpsgd_check_static(int(device), ctypes.c_void_p(stream.cuda_stream))
+    if st:
+        raise WpsgdError(st, "wpsgd_check_static", lib.wpsgd_last_error(None).decode())
 
 
 def _xtype(X) -> int:
@@ -252,6 +283,24 @@ class Context:
                                          self._dev(y, torch.float32, int(so[-1])), so.ctypes.data, ns.ctypes.data,
                                          eta0, sched, lam, loss, seed, self._dev(w0, torch.float32, self.d)),
                  "wpsgd_run_csr")
+
+    def continue_csr(self, row_ptr, col_idx, val, y, shard_off, n_more):
+        import torch
+
+        so, ns = _host_i64(shard_off), _host_i64(n_more)
+        if so.shape[0] != self.k + 1 or ns.shape[0] != self.k:
+            raise ValueError("shard_off must have k+1 entries and n_more k entries")
+        self._ck(self._lib.wpsgd_continue_csr(self._h, self._dev(row_ptr, torch.int64, int(so[-1]) + 1),
+                                              self._dev(col_idx, torch.int32), self._dev(val, torch.float32),
+                                              self._dev(y, torch.float32, int(so[-1])), so.ctypes.data, ns.ctypes.data),
+                 "wpsgd_continue_csr")
+
+    def validate_csr(self, row_ptr, col_idx):
+        import torch
+
+        n_rows = int(row_ptr.numel()) - 1
+        self._ck(self._lib.wpsgd_validate_csr(self._h, self._dev(row_ptr, torch.int64), self._dev(col_idx, torch.int32),
+                                              n_rows, int(col_idx.numel())), "wpsgd_validate_csr")
 
     def run_workload(self, wl):
         """run / run_csr on a workload object (tensors already on the device)."""

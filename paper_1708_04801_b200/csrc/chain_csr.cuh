@@ -23,6 +23,7 @@ struct CsrParams {
   const float* y;
   const long long* shard_off;
   const long long* n_steps;
+  const long long* first;  // steps every node has already run (continued chains), or null
   const long long* idx_off;
   const uint32_t* idx;
   const int* order;
@@ -34,15 +35,17 @@ struct CsrParams {
   int sched;
   float lambda;
   int loss;
+  int resume;  // 1: continue from the models and scales the context holds
   DevStatus* status;
 };
 
-// u rows <- w0 (or zeros), scale <- 1
+// u rows <- w0 (or zeros) unless keep_models, scale <- 1
 __global__ void csr_init_kernel(float* __restrict__ U, double* __restrict__ scale, const float* __restrict__ w0, int k,
-                                long long d) {
+                                long long d, int keep_models) {
   const long long total = (long long)k * d;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x)
-    U[i] = w0 ? w0[i % d] : 0.0f;
+  if (!keep_models)
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x)
+      U[i] = w0 ? w0[i % d] : 0.0f;
   if (blockIdx.x == 0)
     for (int j = threadIdx.x; j < k; j += blockDim.x) scale[j] = 1.0;
 }
@@ -60,7 +63,8 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
   // The scale factor does not depend on the data: s_n = prod_{q<=n} (1 - eta_q lambda). It is advanced in fp64
   // ahead of the chain, together with the rows, and handed to the step as two floats (s before the step, and
   // eta_n / s after it), so that no fp64 division or square root sits on the serial path.
-  double sc = 1.0;  // scale after the last step whose constants have been prepared
+  double sc = p.resume ? p.scale[j] : 1.0;  // scale after the last step whose constants have been prepared
+  const long long first = p.resume ? p.first[j] : 0;
   const double lam = (double)p.lambda, eta0 = (double)p.eta0;
   auto prepare_scalars = [&](long long step0, float& s_before, float& eta_over_s, float& fold) {
     fold = 0.0f;
@@ -69,7 +73,7 @@ __global__ void __launch_bounds__(32) chain_csr_kernel(const CsrParams p) {
       sc = 1.0;
     }
     s_before = (float)sc;
-    const double eta = p.sched == LR_INV_SQRT ? eta0 / sqrt((double)(step0 + 1)) : eta0;
+    const double eta = p.sched == LR_INV_SQRT ? eta0 / sqrt((double)(first + step0 + 1)) : eta0;
     sc *= (1.0 - eta * lam);
     eta_over_s = (float)(eta / sc);
   };

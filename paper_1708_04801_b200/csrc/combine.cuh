@@ -136,4 +136,27 @@ __global__ void __launch_bounds__(256) objective_finish_kernel(const double* __r
   }
 }
 
+// Read-only check of a CSR matrix before it is handed to the chains: row_ptr within [0, nnz] and non-decreasing,
+// every column in [0, d), columns strictly increasing within a row (so no column occurs twice: the sparse update
+// writes every nonzero's model entry once). The first problem found goes to the status word (where = 31 row extents,
+// 32 column range, 33 column order; detail = the row). Nothing is read outside [0, nnz).
+__global__ void validate_csr_kernel(const long long* __restrict__ row_ptr, const int* __restrict__ col_idx, long long n_rows,
+                                    long long nnz, long long d, DevStatus* status) {
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long i = warp0; i < n_rows; i += nwarps) {
+    const long long b = row_ptr[i], e = row_ptr[i + 1];
+    if (b < 0 || e < b || e > nnz) {
+      if (lane == 0) set_status(status, DEV_BOUNDS, 31, i);
+      continue;
+    }
+    for (long long q = b + lane; q < e; q += 32) {
+      const long long c = col_idx[q];
+      if (c < 0 || c >= d) set_status(status, DEV_BOUNDS, 32, i);
+      else if (q > b && (long long)col_idx[q - 1] >= c) set_status(status, DEV_BOUNDS, 33, i);
+    }
+  }
+}
+
 }  // namespace wpsgd

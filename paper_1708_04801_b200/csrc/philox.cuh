@@ -10,11 +10,20 @@
 
 namespace wpsgd {
 
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+// High 32 bits of a 32 x 32 -> 64 bit product, on the device and on the host.
+__host__ __device__ __forceinline__ uint32_t mulhi32(uint32_t a, uint32_t b) {
+#ifdef __CUDA_ARCH__
+  return __umulhi(a, b);
+#else
+  return (uint32_t)(((unsigned long long)a * (unsigned long long)b) >> 32);
+#endif
+}
+
+__host__ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
 #pragma unroll
   for (int i = 0; i < 10; ++i) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    const uint32_t hi0 = mulhi32(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = mulhi32(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
     c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
     k0 += 0x9E3779B9u;
     k1 += 0xBB67AE85u;
@@ -27,7 +36,7 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
 // The n-th example is row pi((n-1) mod m). pi is a 4-round balanced Feistel network on 2w bits (2w = the even
 // bit count >= 2 covering m-1) with cycle walking; round keys = the Philox block at counter (0, 0, node, 1);
 // round function = a 32-bit multiply / xor-shift mixer masked to w bits.
-__device__ __forceinline__ uint32_t mix_round(uint32_t x, uint32_t key) {
+__host__ __device__ __forceinline__ uint32_t mix_round(uint32_t x, uint32_t key) {
   uint32_t h = x ^ key;
   h *= 0x85EBCA6Bu;
   h ^= h >> 13;
@@ -36,9 +45,10 @@ __device__ __forceinline__ uint32_t mix_round(uint32_t x, uint32_t key) {
   return h;
 }
 
-__device__ __forceinline__ uint32_t shuffled_row(const uint4& keys, long long step0 /*0-based*/, uint32_t m) {
+__host__ __device__ __forceinline__ uint32_t shuffled_row(const uint4& keys, long long step0 /*0-based*/, uint32_t m) {
   if (m <= 1u) return 0u;
-  int bits = 32 - __clz((int)(m - 1u));  // smallest bits with 2^bits >= m (m >= 2)
+  int bits = 0;  // smallest bits with 2^bits >= m (m >= 2)
+  while (bits < 32 && ((m - 1u) >> bits) != 0u) ++bits;
   if (bits < 2) bits = 2;
   if (bits & 1) ++bits;
   const int w = bits >> 1;
@@ -63,7 +73,7 @@ __device__ __forceinline__ uint32_t shuffled_row(const uint4& keys, long long st
 
 // Entries of steps b+1 .. b+cnt of node j (shard of m rows) into out[0 .. cnt). sampling 0: one counter value q
 // (four consecutive steps) per (t0 + i * stride); sampling 1: one step per (t0 + i * stride).
-__device__ __forceinline__ void emit_indices(int sampling, uint64_t seed, uint32_t j, long long b, long long cnt, uint32_t m,
+__host__ __device__ __forceinline__ void emit_indices(int sampling, uint64_t seed, uint32_t j, long long b, long long cnt, uint32_t m,
                                              uint32_t* __restrict__ out, long long t0, long long stride) {
   if (sampling == 1) {
     const uint4 keys = philox4x32_10(make_uint4(0u, 0u, j, 1u), (uint32_t)seed, (uint32_t)(seed >> 32));
@@ -78,7 +88,7 @@ __device__ __forceinline__ void emit_indices(int sampling, uint64_t seed, uint32
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const long long s = (q << 2) + e;
-      if (s >= b && s < b + cnt) out[s - b] = __umulhi(w[e], m);  // floor(u m / 2^32)
+      if (s >= b && s < b + cnt) out[s - b] = mulhi32(w[e], m);  // floor(u m / 2^32)
     }
   }
 }

@@ -12,6 +12,7 @@
 
 #include "chain_block.cuh"
 #include "chain_csr.cuh"
+#include "chain_csr_block.cuh"
 #include "chain_mma.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
@@ -62,6 +63,7 @@ struct wpsgd_ctx {
   // options
   int opt_stages = 0;
   int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_cluster = 0;
+  int opt_sparse_variant = 0;  // 0: chosen here, 1: one step per round trip, 2: blocks of steps through a shared-memory cache
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
   int opt_sampling = 0;  // 0: i.i.d. draws, 1: one shuffle per node, cycled
@@ -179,6 +181,19 @@ wpsgd_status weights_host(const long long* n, int k, float eta0, int sched, floa
   if (sum_rT) *sum_rT = tot_raw;
   if (cond) *cond = (2.0 * tot_raw > std::sqrt((double)k) + (double)k) ? 1 : 0;
   return WPSGD_OK;
+}
+
+// Waits for the stream, reads a device status word and maps it; a problem found is cleared after it has been reported.
+wpsgd_status read_status(wpsgd_ctx* c, DevStatus* dev_status, cudaStream_t stream) {
+  DevStatus h;
+  CU_TRY(c, cudaMemcpyAsync(&h, dev_status, sizeof(h), cudaMemcpyDeviceToHost, stream));
+  CU_TRY(c, cudaStreamSynchronize(stream));
+  if (h.code == DEV_OK) return WPSGD_OK;
+  char buf[200];
+  const char* what = h.code == DEV_TIMEOUT ? "a bounded device-side wait gave up" : "a device-side check of the input failed";
+  snprintf(buf, sizeof(buf), "%s: device status %d at %d (detail %lld)", what, h.code, h.where, h.detail);
+  cudaMemsetAsync(dev_status, 0, sizeof(DevStatus), stream);
+  return fail(c, h.code == DEV_TIMEOUT ? WPSGD_ERR_TIMEOUT : WPSGD_ERR_CUDA, buf);
 }
 
 int grid_for(long long work_items, int block, int cap = 148 * 16) {
@@ -642,6 +657,60 @@ wpsgd_status run_dense_common(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, long 
   return WPSGD_OK;
 }
 
+// ---- sparse chain launch ---------------------------------------------------------------------------------
+wpsgd_status run_csr_common(wpsgd_ctx* c, const long long* row_ptr, const int* col_idx, const float* val, const float* y,
+                            const long long* shard_off, const long long* n_steps, const float* w0, bool resume) {
+  Plan pl;
+  std::vector<long long> first = resume ? c->steps_done : std::vector<long long>(c->k, 0);
+  wpsgd_status s = make_plan(c, shard_off, n_steps, first, &pl);
+  if (s != WPSGD_OK) return s;
+  if (pl.total > 0 && (!row_ptr || !col_idx || !val || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "a CSR array or y is NULL");
+  s = upload_plan_and_stream(c, pl);
+  if (s != WPSGD_OK) return s;
+  if (!resume || !c->scaled) {
+    // fresh chains start from w0 with scale 1; chains continued from a dense run keep their models and get scale 1
+    csr_init_kernel<<<grid_for((long long)c->k * c->d, 256), 256, 0, c->stream>>>(c->W, c->scale, w0, c->k, c->d, resume ? 1 : 0);
+    CU_TRY(c, cudaGetLastError());
+    c->launches++;
+  }
+  CsrParams p;
+  p.row_ptr = row_ptr; p.col_idx = col_idx; p.val = val; p.y = y;
+  p.shard_off = c->t_shard_off; p.n_steps = c->t_steps; p.first = c->t_first; p.idx_off = c->t_idx_off; p.idx = c->idx;
+  p.order = c->t_order; p.U = c->W; p.scale = c->scale; p.k = c->k; p.d = c->d;
+  p.eta0 = c->eta0; p.sched = c->sched; p.lambda = c->lambda; p.loss = c->loss; p.resume = resume ? 1 : 0;
+  p.status = c->status;
+  s = timing_begin(c);
+  if (s != WPSGD_OK) return s;
+  if (c->opt_sparse_variant == 1) {
+    const int pf = c->opt_prefetch > 0 ? c->opt_prefetch : 4;
+    if (pf >= 8) chain_csr_kernel<8><<<c->k, 32, 0, c->stream>>>(p);
+    else if (pf >= 4) chain_csr_kernel<4><<<c->k, 32, 0, c->stream>>>(p);
+    else chain_csr_kernel<2><<<c->k, 32, 0, c->stream>>>(p);
+    CU_TRY(c, cudaGetLastError());
+  } else {
+    const size_t smem = sizeof(CsrBlockSmem);
+    auto go = [&](auto kern) -> wpsgd_status {
+      CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      kern<<<c->k, CSRB_THREADS, smem, c->stream>>>(p);
+      CU_TRY(c, cudaGetLastError());
+      return WPSGD_OK;
+    };
+    switch (c->loss) {
+      case WPSGD_LOSS_HINGE: s = go(chain_csr_block_kernel<LOSS_HINGE>); break;
+      case WPSGD_LOSS_LOGISTIC: s = go(chain_csr_block_kernel<LOSS_LOGISTIC>); break;
+      default: s = go(chain_csr_block_kernel<LOSS_SQUARED>); break;
+    }
+    if (s != WPSGD_OK) return s;
+  }
+  c->launches++;
+  s = timing_end(c);
+  if (s != WPSGD_OK) return s;
+  for (int j = 0; j < c->k; ++j) c->steps_done[j] = first[j] + n_steps[j];
+  c->have_run = true;
+  c->scaled = true;
+  return WPSGD_OK;
+}
+
 }  // namespace
 
 // ---- built-in scratch of the entry point that allocates nothing ----------------------------------------
@@ -783,6 +852,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "host_pipeline") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "host_pipeline must be 0 or 1");
     c->opt_host_pipeline = (int)value;
+  } else if (n == "sparse_variant") {
+    if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_variant must be 0, 1 or 2");
+    c->opt_sparse_variant = (int)value;
   } else if (n == "stages") {
     if (value < 0 || value == 1 || value > 8) return fail(c, WPSGD_ERR_INVALID_ARG, "stages must be 0 or 2..8");
     c->opt_stages = (int)value;
@@ -831,7 +903,7 @@ wpsgd_status wpsgd_continue(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, int64_t
                             const int64_t* shard_off, const int64_t* n_more) {
   if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
   if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "continue before run");
-  if (c->scaled) return fail(c, WPSGD_ERR_UNSUPPORTED, "continue is available for dense data only");
+  if (c->scaled) return fail(c, WPSGD_ERR_UNSUPPORTED, "chains started on CSR rows continue with wpsgd_continue_csr");
   DeviceGuard guard(c->device);
   return run_dense_common(c, X, xt, ld_elems, y, (const long long*)shard_off, (const long long*)n_more, nullptr, true);
 }
@@ -845,34 +917,17 @@ wpsgd_status wpsgd_run_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* 
   if (s != WPSGD_OK) return s;
   c->eta0 = eta0; c->sched = (int)sched; c->lambda = lambda; c->loss = (int)loss; c->seed = seed;
   c->have_run = false;
-  Plan pl;
-  s = make_plan(c, (const long long*)shard_off, (const long long*)n_steps, std::vector<long long>(c->k, 0), &pl);
-  if (s != WPSGD_OK) return s;
-  if (pl.total > 0 && (!row_ptr || !col_idx || !val || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "a CSR array or y is NULL");
-  s = upload_plan_and_stream(c, pl);
-  if (s != WPSGD_OK) return s;
-  csr_init_kernel<<<grid_for((long long)c->k * c->d, 256), 256, 0, c->stream>>>(c->W, c->scale, w0, c->k, c->d);
-  CU_TRY(c, cudaGetLastError());
-  c->launches++;
-  CsrParams p;
-  p.row_ptr = (const long long*)row_ptr; p.col_idx = col_idx; p.val = val; p.y = y;
-  p.shard_off = c->t_shard_off; p.n_steps = c->t_steps; p.idx_off = c->t_idx_off; p.idx = c->idx;
-  p.order = c->t_order; p.U = c->W; p.scale = c->scale; p.k = c->k; p.d = c->d;
-  p.eta0 = eta0; p.sched = (int)sched; p.lambda = lambda; p.loss = (int)loss; p.status = c->status;
-  s = timing_begin(c);
-  if (s != WPSGD_OK) return s;
-  const int pf = c->opt_prefetch > 0 ? c->opt_prefetch : 4;
-  if (pf >= 8) chain_csr_kernel<8><<<c->k, 32, 0, c->stream>>>(p);
-  else if (pf >= 4) chain_csr_kernel<4><<<c->k, 32, 0, c->stream>>>(p);
-  else chain_csr_kernel<2><<<c->k, 32, 0, c->stream>>>(p);
-  CU_TRY(c, cudaGetLastError());
-  c->launches++;
-  s = timing_end(c);
-  if (s != WPSGD_OK) return s;
-  for (int j = 0; j < c->k; ++j) c->steps_done[j] = n_steps[j];
-  c->have_run = true;
-  c->scaled = true;
-  return WPSGD_OK;
+  return run_csr_common(c, (const long long*)row_ptr, col_idx, val, y, (const long long*)shard_off,
+                        (const long long*)n_steps, w0, false);
+}
+
+wpsgd_status wpsgd_continue_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                                const float* y, const int64_t* shard_off, const int64_t* n_more) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->have_run) return fail(c, WPSGD_ERR_STATE, "continue before run");
+  DeviceGuard guard(c->device);
+  return run_csr_common(c, (const long long*)row_ptr, col_idx, val, y, (const long long*)shard_off,
+                        (const long long*)n_more, nullptr, true);
 }
 
 wpsgd_status wpsgd_get_weights(wpsgd_ctx* c, double r, double* weights, int* cond_holds) {
@@ -888,6 +943,49 @@ wpsgd_status wpsgd_weights(const int64_t* n_steps, int32_t k, float eta0, wpsgd_
   std::string why;
   wpsgd_status s = weights_host((const long long*)n_steps, k, eta0, (int)sched, lambda, r, weights, cond_holds, sum_rT, &why);
   return s == WPSGD_OK ? s : fail(nullptr, s, why);
+}
+
+wpsgd_status wpsgd_span_valid(const int64_t* n_steps, int32_t k, float eta0, float lambda, double r, int64_t span,
+                              double* lhs, int* holds) {
+  if (span < 0) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "span_valid: span must be >= 0");
+  if (!((double)eta0 * (double)lambda < 1.0) || !(eta0 >= 0.0f) || !(lambda >= 0.0f))
+    return fail(nullptr, WPSGD_ERR_INVALID_ARG, "span_valid: need eta0 >= 0, lambda >= 0, eta0 * lambda < 1");
+  if (!n_steps || k < 1) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "span_valid: null argument or k < 1");
+  std::string why;
+  std::vector<double> lg;
+  wpsgd_status s = log_rates((const long long*)n_steps, k, (double)eta0, WPSGD_LR_CONST, (double)lambda, r, &lg, &why);
+  if (s != WPSGD_OK) return fail(nullptr, s, why);
+  // log of sum_j r^{T_j}, summed from the largest term
+  const double mx = *std::max_element(lg.begin(), lg.end());
+  double tot = 0.0;
+  for (int j = 0; j < k; ++j) tot += std::exp(lg[j] - mx);
+  const double log_lhs = std::log((double)k) - (mx + std::log(tot)) + (double)span * std::log1p(-(double)eta0 * (double)lambda);
+  const double v = std::exp(log_lhs);
+  if (lhs) *lhs = v;
+  if (holds) *holds = log_lhs < 0.0 ? 1 : 0;
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_sample_indices_host(uint64_t seed, int32_t node, int64_t m, int64_t n_begin, int64_t count,
+                                       int32_t sampling, uint32_t* out) {
+  if (node < 0 || m < 1 || m > 0xFFFFFFFFll || n_begin < 0 || count < 0 || (sampling != 0 && sampling != 1))
+    return fail(nullptr, WPSGD_ERR_INVALID_ARG,
+                "sample_indices_host: need node >= 0, 1 <= m < 2^32, n_begin >= 0, count >= 0, sampling 0 or 1");
+  if (count == 0) return WPSGD_OK;
+  if (!out) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "out is NULL");
+  emit_indices(sampling, seed, (uint32_t)node, n_begin, count, (uint32_t)m, out, 0, 1);  // the kernels' own function
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_validate_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* col_idx, int64_t n_rows, int64_t nnz) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (n_rows < 0 || nnz < 0 || !row_ptr || (nnz > 0 && !col_idx)) return fail(c, WPSGD_ERR_INVALID_ARG, "validate_csr: bad argument");
+  if (n_rows == 0) return WPSGD_OK;
+  DeviceGuard guard(c->device);
+  validate_csr_kernel<<<grid_for(n_rows, 8), 256, 0, c->stream>>>((const long long*)row_ptr, col_idx, n_rows, nnz, c->d, c->status);
+  CU_TRY(c, cudaGetLastError());
+  c->launches++;
+  return WPSGD_OK;
 }
 
 wpsgd_status wpsgd_combine(wpsgd_ctx* c, double r, float* v_out) {
@@ -1166,14 +1264,22 @@ wpsgd_status wpsgd_solve_static(int device, void* cuda_stream, const void* X, wp
 wpsgd_status wpsgd_check(wpsgd_ctx* c) {
   if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
   DeviceGuard guard(c->device);
-  DevStatus h;
-  CU_TRY(c, cudaMemcpyAsync(&h, c->status, sizeof(h), cudaMemcpyDeviceToHost, c->stream));
-  CU_TRY(c, cudaStreamSynchronize(c->stream));
-  if (h.code == DEV_OK) return WPSGD_OK;
-  char buf[160];
-  snprintf(buf, sizeof(buf), "device status %d at %d (detail %lld)", h.code, h.where, h.detail);
-  cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream);
-  return fail(c, h.code == DEV_TIMEOUT ? WPSGD_ERR_TIMEOUT : WPSGD_ERR_CUDA, buf);
+  return read_status(c, c->status, c->stream);
+}
+
+wpsgd_status wpsgd_check_static(int device, void* cuda_stream) {
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    return fail(nullptr, WPSGD_ERR_CUDA, "no CUDA device available");
+  }
+  if (device < 0 || device >= ndev || device >= kStaticMaxDevices)
+    return fail(nullptr, WPSGD_ERR_INVALID_ARG, "check_static: device index out of range");
+  DeviceGuard guard(device);
+  unsigned char* base = nullptr;
+  wpsgd_status s = static_scratch_base(device, &base);
+  if (s != WPSGD_OK) return s;
+  return read_status(nullptr, (DevStatus*)(base + StaticLayout().status), (cudaStream_t)cuda_stream);
 }
 
 int64_t wpsgd_launch_count(const wpsgd_ctx* c) { return c ? c->launches : 0; }

@@ -108,9 +108,42 @@ def test_validity_condition_of_averaging_every_span(wpsgd_lib):
     r = 1.0 - float(np.float32(0.1)) * float(np.float32(0.01))
     tot = 2 + 2 * r ** 1000
     for span, want in ((100, (4 / tot) * r ** 100), (1000, (4 / tot) * r ** 1000)):
-        holds, lhs = P.averaging_span_valid(n, 0.1, 0.01, span)
+        holds, lhs = P.span_valid(n, 0.1, 0.01, span)
         assert lhs == pytest.approx(want, rel=1e-9)
         assert holds == (want < 1.0)
-    assert P.averaging_span_valid(n, 0.1, 0.01, 100)[0] is False   # a short span cannot make up for the delays
-    assert P.averaging_span_valid(n, 0.1, 0.01, 1000)[0] is True
-    assert P.averaging_span_valid([50, 50, 50], 0.1, 0.01, 1)[0] is True   # balanced: any span is valid
+    assert P.span_valid(n, 0.1, 0.01, 100)[0] is False   # a short span cannot make up for the delays
+    assert P.span_valid(n, 0.1, 0.01, 1000)[0] is True
+    assert P.span_valid([50, 50, 50], 0.1, 0.01, 1)[0] is True   # balanced: any span is valid
+    with pytest.raises(P.WpsgdError) as e:
+        P.span_valid(n, 0.1, 0.01, -1)
+    assert e.value.status_name == "INVALID_ARG"
+    # a caller-given rate (Eq. 8) enters the sum, the contraction per step stays 1 - eta lambda
+    holds, lhs = P.span_valid(n, 0.1, 0.01, 500, r=0.9995)
+    assert lhs == pytest.approx((4 / (2 + 2 * 0.9995 ** 1000)) * r ** 500, rel=1e-9)
+
+
+@pytest.mark.parametrize("seed,node,m,n_begin,count", [
+    (0, 0, 4096, 0, 1000), (12345678901234567, 3, 1, 0, 17), (7, 1023, (1 << 32) - 1, 5, 64),
+    (2, 9, 65536, (1 << 34) + 3, 33), (3, 2, 3, 1, 2), (1, 0, 100, 7, 0),
+])
+@pytest.mark.parametrize("sampling", [0, 1])
+def test_host_sample_stream_is_bit_exact(wpsgd_lib, seed, node, m, n_begin, count, sampling):
+    """The library's host-side stream (the function its kernels call) against the checker's own Philox / shuffle."""
+    import paper_1708_04801_b200 as P
+
+    got = P.sample_indices_host(seed, node, m, n_begin, count, sampling)
+    oracle.set_sampling(sampling)
+    try:
+        want = oracle.sample_indices(seed, node, m, n_begin, count)
+    finally:
+        oracle.set_sampling(0)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_host_sample_stream_rejects_bad_input(wpsgd_lib):
+    import paper_1708_04801_b200 as P
+
+    for args in ((0, -1, 10, 0, 5, 0), (0, 0, 0, 0, 5, 0), (0, 0, 1 << 32, 0, 5, 0), (0, 0, 10, -1, 5, 0), (0, 0, 10, 0, 5, 2)):
+        with pytest.raises(P.WpsgdError) as e:
+            P.sample_indices_host(*args)
+        assert e.value.status_name == "INVALID_ARG"

@@ -572,24 +572,158 @@ def test_solve_host_pipelined_equals_device_path(P, d, bf16, k, pipeline):
 
 
 # ---- sparse path --------------------------------------------------------------------------------------------
+# sparse_variant 1: one step per round trip to the model in global memory; 2 (the default): blocks of steps run in a
+# shared-memory cache of the model entries they touch
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
-@pytest.mark.parametrize("prefetch", [2, 4, 8])
-def test_csr_losses_and_prefetch_depths(P, loss, prefetch):
+@pytest.mark.parametrize("variant,prefetch", [(1, 2), (1, 4), (1, 8), (2, 0)])
+def test_csr_losses_and_kernels(P, loss, variant, prefetch):
     wl = wi.config4(k=5, d=4096, m=300, base_steps=700, mean_nnz=30.0)
     wl.loss = loss
     if loss == SQUARED:
         wl.eta0 = 0.05
     wl.w0 = torch.full((4096,), 0.01)
-    assert_parity(P, wl, {"prefetch": prefetch})
+    assert_parity(P, wl, {"sparse_variant": variant, "prefetch": prefetch})
 
 
-def test_csr_long_rows_and_strong_regulariser(P):
+@pytest.mark.parametrize("variant", [1, 2])
+def test_csr_long_rows_and_strong_regulariser(P, variant):
     # rows with up to 128 nonzeros (beyond the 64 kept in registers); eta*lambda large enough that the
     # scale factor is folded back into the model several times
     wl = wi.config4(k=3, d=512, m=64, base_steps=400, mean_nnz=90.0, max_nnz=128)
     wl.sched, wl.eta0, wl.lam = 0, 0.5, 0.5  # (1 - 0.25)^400 ~ 1e-50
     wl.w0 = torch.full((512,), 1.0)
-    assert_parity(P, wl)
+    assert_parity(P, wl, {"sparse_variant": variant})
+
+
+@pytest.mark.parametrize("n_steps", [(1, 63, 64), (65, 127, 128), (129, 0, 200), (333, 250, 3)])
+@pytest.mark.parametrize("mean_nnz", [8.0, 100.0])
+def test_csr_block_kernel_block_boundaries(P, n_steps, mean_nnz):
+    # short rows: a block ends after 64 steps; long rows: it ends when its 4096 table entries are used up
+    wl = wi.config4(k=3, d=2048, m=96, base_steps=10, mean_nnz=mean_nnz, max_nnz=128)
+    wl.n_steps = np.array(n_steps, dtype=np.int64)
+    wl.w0 = torch.full((2048,), 0.02)
+    assert_parity(P, wl, {"sparse_variant": 2})
+
+
+def _rows_with_given_lengths(lengths, d, seed):
+    """Hand-built CSR rows of the given lengths: distinct sorted random columns, values 1/sqrt(nnz), labels +-1."""
+    g = torch.Generator().manual_seed(seed)
+    cols, vals = [], []
+    for n in lengths:
+        c, _ = torch.sort(torch.randperm(d, generator=g)[:n])
+        cols.append(c.to(torch.int32))
+        vals.append(torch.full((n,), 1.0 / np.sqrt(max(n, 1))))
+    rp = torch.zeros(len(lengths) + 1, dtype=torch.int64)
+    rp[1:] = torch.cumsum(torch.tensor(lengths), 0)
+    y = torch.where(torch.rand(len(lengths), generator=g) < 0.5, 1.0, -1.0)
+    return rp, torch.cat(cols), torch.cat(vals), y
+
+
+@pytest.mark.parametrize("loss", [HINGE, SQUARED])
+def test_csr_rows_longer_than_the_block_tables(P, loss):
+    # rows of 5000 and 6000 nonzeros do not fit the 4096 table entries of a block: such a step is run on global
+    # memory, between ordinary blocks of short rows
+    d = 8192
+    lengths = [5000, 12, 30, 6000, 7, 4096, 4097, 64, 1, 0, 33, 65]
+    rp, ci, va, y = _rows_with_given_lengths(lengths, d, 11)
+    wl = wi.Workload("long", 2, d, np.array([0, 6, 12]), np.array([150, 90]), 0.2, 1, 0.01, loss, 5, y, row_ptr=rp,
+                     col_idx=ci, val=va, w0=torch.full((d,), 0.01))
+    assert_parity(P, wl, {"sparse_variant": 2})
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_continue_csr_equals_one_run(P, variant):
+    wl_cpu = wi.config4(k=3, d=4096, m=128, base_steps=10, mean_nnz=30.0)
+    wl_cpu.n_steps = np.array([203, 101, 50], dtype=np.int64)
+    wl_cpu.lam = 0.01
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("sparse_variant", variant)
+        ctx.run_workload(wl)
+        full = ctx.get_models().cpu().numpy()
+        cuts = [np.array([50, 50, 50]), np.array([1, 1, 0]), np.array([152, 50, 0])]
+        ctx.run_csr(wl.row_ptr, wl.col_idx, wl.val, wl.y, wl.shard_off, cuts[0], wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        for c in cuts[1:]:
+            ctx.continue_csr(wl.row_ptr, wl.col_idx, wl.val, wl.y, wl.shard_off, c)
+        seg = ctx.get_models().cpu().numpy()
+        wts, _ = ctx.get_weights()
+        ctx.check()
+    if variant == 1:
+        np.testing.assert_array_equal(seg, full)  # same arithmetic in the same order
+    else:
+        # the fp64 scale is a product over the steps of a block, so cutting the chain changes its last bits only
+        for j in range(wl.k):
+            assert rel_l2(seg[j], full[j]) <= 1e-6
+    owts, _, _ = oracle.weights(wl_cpu.n_steps, wl_cpu.eta0, wl_cpu.sched, wl_cpu.lam)
+    np.testing.assert_allclose(wts, owts, rtol=1e-12)
+    oW = oracle.run_csr(wl_cpu.row_ptr, wl_cpu.col_idx, wl_cpu.val, wl_cpu.y, wl_cpu.shard_off, wl_cpu.n_steps, wl_cpu.d,
+                        wl_cpu.eta0, wl_cpu.sched, wl_cpu.lam, wl_cpu.loss, wl_cpu.seed)
+    for j in range(wl.k):
+        assert rel_l2(seg[j], oW[j]) <= TOL[wl_cpu.loss]
+
+
+def test_periodic_weighted_averaging_on_csr_rows(P):
+    # average every span of fastest-node steps, broadcast, continue: the paper's bucket-style WP-SGD on sparse rows.
+    # The checker runs the same schedule on the densified rows (its dense loop can start from a given model and step).
+    wl = wi.config4(k=4, d=256, m=64, base_steps=10, mean_nnz=12.0, max_nnz=32)
+    wl.loss, wl.sched, wl.eta0, wl.lam = LOGISTIC, 0, 0.1, 0.01
+    span_steps = [np.array([40, 20, 10, 40]), np.array([40, 20, 10, 40]), np.array([40, 20, 10, 40])]
+    dev = wl.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.run_csr(dev.row_ptr, dev.col_idx, dev.val, dev.y, wl.shard_off, span_steps[0], wl.eta0, wl.sched, wl.lam,
+                    wl.loss, wl.seed)
+        for seg in span_steps[1:]:
+            ctx.set_models(ctx.combine())
+            ctx.continue_csr(dev.row_ptr, dev.col_idx, dev.val, dev.y, wl.shard_off, seg)
+        v = ctx.combine().cpu().numpy()
+        ctx.check()
+    dn = wi.densify(wl)
+    W = oracle.run_dense(dn.X, dn.y, wl.shard_off, span_steps[0], wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    done = span_steps[0].copy()
+    for seg in span_steps[1:]:
+        wts, _, _ = oracle.weights(done, wl.eta0, wl.sched, wl.lam)
+        vv = oracle.combine(W, wts)
+        Wn = np.zeros_like(W)
+        for j in range(wl.k):
+            only = np.zeros(wl.k, dtype=np.int64)
+            only[j] = seg[j]
+            Wn[j] = oracle.run_dense(dn.X, dn.y, wl.shard_off, only, wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed,
+                                     step_begin=int(done[j]),
+                                     W_resume=np.tile(vv.astype(np.float32).astype(np.float64), (wl.k, 1)))[j]
+        W = Wn
+        done = done + seg
+    wts, _, _ = oracle.weights(done, wl.eta0, wl.sched, wl.lam)
+    assert rel_l2(v, oracle.combine(W, wts)) <= 1e-4
+
+
+def test_validate_csr_accepts_good_input_and_names_the_bad_row(P):
+    # the malformed arrays below are only ever read by the validator (which reads nothing outside [0, nnz)); they
+    # are never handed to a chain kernel
+    good = wi.config4(k=2, d=512, m=40, base_steps=10, mean_nnz=9.0, max_nnz=20).to("cuda")
+    with P.Context(2, 512) as ctx:
+        ctx.validate_csr(good.row_ptr, good.col_idx)
+        ctx.check()
+        nnz = int(good.col_idx.numel())
+        row7 = slice(int(good.row_ptr[7]), int(good.row_ptr[8]))
+        assert row7.stop - row7.start >= 2
+        cases = []
+        bad = good.col_idx.clone(); bad[row7.start] = 512            # column == d
+        cases.append((good.row_ptr, bad, "detail 7"))
+        bad = good.col_idx.clone(); bad[row7.start + 1] = -3          # negative column
+        cases.append((good.row_ptr, bad, "detail 7"))
+        bad = good.col_idx.clone(); bad[row7.start + 1] = bad[row7.start]   # a column twice in a row
+        cases.append((good.row_ptr, bad, "detail 7"))
+        rp = good.row_ptr.clone(); rp[5] = rp[6] + 1                  # row 4 ends after row 5 starts: row 5 runs backwards
+        cases.append((rp, good.col_idx, "detail 5"))
+        rp = good.row_ptr.clone(); rp[-1] = nnz + 10                  # last row claims entries beyond the arrays
+        cases.append((rp, good.col_idx, f"detail {rp.numel() - 2}"))
+        for rp_, ci_, where in cases:
+            ctx.validate_csr(rp_, ci_)
+            with pytest.raises(P.WpsgdError) as e:
+                ctx.check()
+            assert e.value.status_name == "CUDA" and where in str(e.value), str(e.value)
+        ctx.validate_csr(good.row_ptr, good.col_idx)  # the context is clean again
+        ctx.check()
 
 
 def test_csr_equals_dense_kernels_on_densified_rows(P):

@@ -257,6 +257,27 @@ def test_csr_scaled_form_equals_literal(loss):
     np.testing.assert_array_equal(one, b[2])
 
 
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+def test_csr_scaled_form_folds_its_scale_back_and_still_equals_literal(loss):
+    """eta*lambda = 0.5 for 400 steps: the scale factor passes 1e-100 after 333 steps (0.5^333 = 5.7e-101), so the
+    scaled form multiplies it back into u on the way; the literal O(d) form has no scale at all."""
+    wl = _small_sparse(loss)
+    wl.sched, wl.eta0, wl.lam = 0, 0.5, 1.0
+    wl.n_steps = np.array([400, 340, 5], dtype=np.int64)[: wl.k] if wl.k <= 3 else np.array(
+        [400, 340, 5] + [332] * (wl.k - 3), dtype=np.int64)
+    assert 0.5 ** int(wl.n_steps.max()) < 1e-100
+    w0 = torch.full((wl.d,), 2.0)
+    a = oracle.run_csr(wl.row_ptr, wl.col_idx, wl.val, wl.y, wl.shard_off, wl.n_steps, wl.d, wl.eta0, wl.sched,
+                       wl.lam, loss, wl.seed, w0, literal=True)
+    b = oracle.run_csr(wl.row_ptr, wl.col_idx, wl.val, wl.y, wl.shard_off, wl.n_steps, wl.d, wl.eta0, wl.sched,
+                       wl.lam, loss, wl.seed, w0, literal=False)
+    for j in range(wl.k):
+        assert np.linalg.norm(a[j]) > 0
+        assert np.linalg.norm(a[j] - b[j]) <= 1e-11 * np.linalg.norm(a[j]), j
+    # and the chains really went through the branch: untouched coordinates carry w0 * 0.5^n, far below 1e-100
+    assert 0 < np.abs(a[0]).min() < 1e-100
+
+
 # ---- Eq. 6 / Eq. 8 weights, Eq. 7 / Eq. 9 condition --------------------------------------------------
 def _decimal_weights(n_steps, r):
     getcontext().prec = 60
