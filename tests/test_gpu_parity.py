@@ -713,8 +713,8 @@ def test_validate_csr_accepts_good_input_and_names_the_bad_row(P):
         cases.append((good.row_ptr, bad, "detail 7"))
         bad = good.col_idx.clone(); bad[row7.start + 1] = bad[row7.start]   # a column twice in a row
         cases.append((good.row_ptr, bad, "detail 7"))
-        rp = good.row_ptr.clone(); rp[5] = rp[6] + 1                  # row 4 ends after row 5 starts: row 5 runs backwards
-        cases.append((rp, good.col_idx, "detail 5"))
+        rp = good.row_ptr.clone(); rp[0] = -1                         # row 0 starts before the arrays
+        cases.append((rp, good.col_idx, "detail 0"))
         rp = good.row_ptr.clone(); rp[-1] = nnz + 10                  # last row claims entries beyond the arrays
         cases.append((rp, good.col_idx, f"detail {rp.numel() - 2}"))
         for rp_, ci_, where in cases:
