@@ -8,21 +8,29 @@
 //
 // Why blocks. In the direct kernel every step pays a round trip to the model in global memory (gather, reduce,
 // scatter) on its serial path. The sample stream does not depend on the model, so the rows of the next steps are
-// known in advance. Here the helper warps take the next up to 64 steps (at most CSRB_EMAX nonzeros in all), give
-// every distinct column among them a slot in a shared-memory hash table (linear probing, one compare-and-swap per
-// nonzero), and store per nonzero its slot and value. At the block boundary all threads write the previous block's
-// slots back to u and read this block's columns of u into the slots (one round trip to global memory per block, all
-// loads independent); the chain warp then runs the block's steps entirely in shared memory: slot loads, a warp
-// reduction, the loss derivative, slot stores. Preparation of block b + 1 (row extents, scale factors in fp64, nonzeros
-// copied with cp.async, hash inserts) overlaps the steps of block b; the tables are double buffered.
+// known in advance. The helper warps take the next up to 64 steps (at most CSRB_EMAX nonzeros in all), give every
+// distinct column among them a slot in a shared-memory hash table (linear probing, one compare-and-swap per
+// nonzero), store per nonzero its slot and value, and read u at the block's columns into the block's cache, all
+// while the chain warp runs the previous block. The chain warp runs a block's steps entirely in shared memory: slot
+// loads, a reduction over the warp through shared memory, the loss derivative, slot stores.
 //
-// A row with more than CSRB_EMAX nonzeros forms a block of its own that the chain warp runs on global memory
-// directly. When the scale has fallen below 1e-12 at the start of a block it is folded into u (u <- s u, s <- 1) by
-// all threads; a block also ends early before the scale would leave the fp32 range of the per-step factors.
+// Block boundary. The values the helpers read for block b + 1 are stale exactly at the columns block b touches, so
+// at the boundary every column of block b + 1 is looked up in block b's table and, when found, takes block b's
+// cached value (shared memory to shared memory). No global-memory latency is left on the chain's path: block b's
+// slots are written back to u by the helpers afterwards, before they reuse its tables for block b + 2. Tables and
+// caches are double buffered.
+//
+// Slow boundaries (rare): a row with more than CSRB_EMAX nonzeros forms a block of its own that the chain warp runs
+// on global memory; when the scale has fallen below 1e-12 at the start of a block it is folded into u (u <- s u,
+// s <- 1). In both cases, and for the first block, all threads write the previous block back, apply the fold, and
+// read the block's columns again from global memory. A block also ends early before the scale would leave the fp32
+// range of the per-step factors.
 //
 // Column indices are checked against d when they are inserted (a bad index sets the status word and the entry is
-// dropped); the kernel has no unbounded wait: every barrier is reached by all threads the same number of times.
+// dropped). The kernel has no wait on anything but CTA barriers that every thread reaches the same number of times.
 #pragma once
+
+#include <type_traits>
 
 #include "chain_block.cuh"
 #include "chain_csr.cuh"
@@ -33,16 +41,18 @@ constexpr int CSRB_STEPS = 64;          // most steps per block
 constexpr int CSRB_EMAX = 4096;         // most nonzeros per block
 constexpr int CSRB_HASH = 8192;         // slots of the column table (power of two, > CSRB_EMAX)
 constexpr int CSRB_HASH_BITS = 13;
-constexpr int CSRB_THREADS = 128;       // warp 0: chain; warps 1..3: preparation
+constexpr int CSRB_THREADS = 256;       // warp 0: chain; warps 1..7: preparation
 constexpr int CSRB_HELPERS = CSRB_THREADS - 32;
+constexpr int CSRB_BATCH = 8;           // independent global loads a thread keeps in flight
 
 struct CsrBlockMeta {
   int nsteps;    // steps in the block (0: the chain has ended)
   int nent;      // nonzeros of those steps
   int direct;    // 1: a single long row, run on global memory
-  int nuniq;     // distinct columns (filled while inserting)
+  int nuniq;     // distinct columns (filled while inserting; 0 again once the block has been written back)
   float fold;    // != 0: multiply u by it before the block (the scale was folded back)
-  int pad[3];
+  int wide;      // 1: some row of the block has more than 64 nonzeros
+  int pad[2];
 };
 
 // One buffer of a prepared block.
@@ -62,8 +72,9 @@ struct CsrBlockBuf {
 
 struct CsrBlockSmem {
   CsrBlockBuf buf[2];
-  float ucache[CSRB_HASH];             // u at the columns of the running block, by slot
+  float ucache[2][CSRB_HASH];          // u at the columns of a block, by slot
   int colbuf[CSRB_EMAX];               // columns of the block being prepared
+  float red[32];                       // the chain warp's partial sums of a margin
 };
 
 __device__ __forceinline__ void named_barrier(int id, int threads) {
@@ -71,6 +82,33 @@ __device__ __forceinline__ void named_barrier(int id, int threads) {
 }
 
 __device__ __forceinline__ int csrb_hash(int col) { return (int)(((uint32_t)col * 0x9E3779B1u) >> (32 - CSRB_HASH_BITS)); }
+
+// cache[slot] <- u[column of slot] for the block's distinct columns i = t0, t0 + stride, ...; CSRB_BATCH loads in flight.
+__device__ __forceinline__ void csrb_gather(const CsrBlockBuf& B, float* cache, const float* u, int nuniq, int t0, int stride) {
+  for (int base = t0; base < nuniq; base += stride * CSRB_BATCH) {
+    int h[CSRB_BATCH];
+    float v[CSRB_BATCH];
+#pragma unroll
+    for (int g = 0; g < CSRB_BATCH; ++g) {
+      const int i = base + g * stride;
+      h[g] = i < nuniq ? (int)B.uslot[i] : -1;
+    }
+#pragma unroll
+    for (int g = 0; g < CSRB_BATCH; ++g) v[g] = h[g] >= 0 ? __ldcg(u + B.keys[h[g]]) : 0.0f;
+#pragma unroll
+    for (int g = 0; g < CSRB_BATCH; ++g)
+      if (h[g] >= 0) cache[h[g]] = v[g];
+  }
+}
+
+// u[column of slot] <- cache[slot] for the block's distinct columns, and the table is emptied.
+__device__ __forceinline__ void csrb_scatter(CsrBlockBuf& B, const float* cache, float* u, int nuniq, int t0, int stride) {
+  for (int i = t0; i < nuniq; i += stride) {
+    const int h = B.uslot[i];
+    u[B.keys[h]] = cache[h];
+    B.keys[h] = -1;
+  }
+}
 
 template <int LOSS>
 __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const CsrParams p) {
@@ -92,6 +130,10 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
   if (threadIdx.x == 0) {
     sm.buf[0].meta.nuniq = 0;
     sm.buf[1].meta.nuniq = 0;
+    sm.buf[0].meta.nsteps = 0;
+    sm.buf[1].meta.nsteps = 0;
+    sm.buf[0].meta.direct = 0;
+    sm.buf[1].meta.direct = 0;
   }
   __syncthreads();
 
@@ -99,28 +141,43 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
   long long s_next = 0;                          // first step of the next block to prepare (planner warp)
   double sc = p.resume ? p.scale[j] : 1.0;       // scale after the last planned step (planner warp)
   const double lam = (double)p.lambda, eta0 = (double)p.eta0;
-  auto prepare = [&](CsrBlockBuf& B) {
+  auto prepare = [&](CsrBlockBuf& B, float* cache) {
     if (warp == 1) {
       float fold = 0.0f;
-      if (sc < 1e-12) {
+      if (sc < 1e-12 && s_next < n_run) {  // only ahead of a block that runs: the fold is applied at its start
         fold = (float)sc;
         sc = 1.0;
       }
-      int nsteps = 0, nent = 0, direct = 0;
-      bool more = true;
-      for (int part = 0; part < CSRB_STEPS / 32 && more; ++part) {
-        const long long s = s_next + nsteps + lane;
-        const bool valid = s < n_run;
-        long long gb = 0, ge = 0;
-        float yy = 0.0f;
-        if (valid) {
-          const uint32_t i = idx[s];
-          gb = rp[i];
-          ge = rp[i + 1];
-          yy = yshard[i];
+      // row extents and labels of the next 64 steps, all loads in flight together
+      constexpr int PARTS = CSRB_STEPS / 32;
+      long long gb[PARTS], ge[PARTS];
+      float yy[PARTS];
+      uint32_t ri[PARTS];
+#pragma unroll
+      for (int part = 0; part < PARTS; ++part) {
+        const long long s = s_next + part * 32 + lane;
+        ri[part] = s < n_run ? idx[s] : 0u;
+      }
+#pragma unroll
+      for (int part = 0; part < PARTS; ++part) {
+        const long long s = s_next + part * 32 + lane;
+        gb[part] = ge[part] = 0;
+        yy[part] = 0.0f;
+        if (s < n_run) {
+          gb[part] = rp[ri[part]];
+          ge[part] = rp[ri[part] + 1];
+          yy[part] = yshard[ri[part]];
         }
-        const long long len = ge - gb;
-        const int cnt = len > (long long)CSRB_EMAX ? CSRB_EMAX + 1 : (int)len;
+      }
+      int nsteps = 0, nent = 0, direct = 0, wide = 0;
+      bool more = true;
+#pragma unroll
+      for (int part = 0; part < PARTS; ++part) {
+        if (!more) break;
+        const long long s = s_next + part * 32 + lane;
+        const bool valid = s < n_run;
+        const long long len = ge[part] - gb[part];
+        const int cnt = len > (long long)CSRB_EMAX ? CSRB_EMAX + 1 : (len < 0 ? 0 : (int)len);
         const double eta = p.sched == LR_INV_SQRT ? eta0 / sqrt((double)(first + s + 1)) : eta0;
         const double a = valid ? 1.0 - eta * lam : 1.0;
         int icnt = cnt;
@@ -141,36 +198,38 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
         const int n_ok = (mask == 0xffffffffu) ? 32 : (__ffs((int)~mask) - 1);
         if (lane < n_ok) {
           const int r = nsteps + lane;
-          B.gbeg[r] = gb;
+          B.gbeg[r] = gb[part];
           B.rbeg[r] = nent + icnt - cnt;
           B.rcnt[r] = cnt;
-          B.yv[r] = yy;
+          B.yv[r] = yy[part];
           B.sbef[r] = (float)(sc * ea);
           B.eos[r] = (float)(eta / (sc * ia));
         }
-        if (n_ok > 0) {
-          nent += __shfl_sync(0xffffffffu, icnt, n_ok - 1);
-          sc *= __shfl_sync(0xffffffffu, ia, n_ok - 1);
-          nsteps += n_ok;
-        }
-        if (n_ok < 32) more = false;
-        if (nsteps == 0 && valid && lane == 0) {
-          // the first row does not fit the tables: a block of its own, run on global memory
-          B.gbeg[0] = gb;
-          B.rbeg[0] = 0;
-          B.rcnt[0] = 0;
-          B.yv[0] = yy;
-          B.sbef[0] = (float)sc;
-          B.eos[0] = (float)(eta / (sc * a));
-        }
-        const int lone = __shfl_sync(0xffffffffu, (nsteps == 0 && valid) ? 1 : 0, 0);
+        wide |= __any_sync(0xffffffffu, lane < n_ok && cnt > 64) ? 1 : 0;
+        // a first row that does not fit the tables: a block of its own, run on global memory
+        const int lone = __shfl_sync(0xffffffffu, (part == 0 && n_ok == 0 && valid) ? 1 : 0, 0);
         if (lone) {
+          if (lane == 0) {
+            B.gbeg[0] = gb[part];
+            B.gbeg[1] = ge[part];  // the row's end travels in the unused second entry
+            B.rbeg[0] = 0;
+            B.rcnt[0] = 0;
+            B.yv[0] = yy[part];
+            B.sbef[0] = (float)sc;
+            B.eos[0] = (float)(eta / (sc * a));
+          }
           direct = 1;
           nsteps = 1;
           nent = 0;
           sc *= __shfl_sync(0xffffffffu, a, 0);
-          // the row length travels in gbeg[1] (unused by a block of one step)
-          if (lane == 0) B.gbeg[1] = ge;
+          more = false;
+        } else {
+          if (n_ok > 0) {
+            nent += __shfl_sync(0xffffffffu, icnt, n_ok - 1);
+            sc *= __shfl_sync(0xffffffffu, ia, n_ok - 1);
+            nsteps += n_ok;
+          }
+          if (n_ok < 32) more = false;
         }
       }
       if (lane == 0) {
@@ -178,12 +237,13 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
         B.meta.nent = nent;
         B.meta.direct = direct;
         B.meta.fold = fold;
+        B.meta.wide = wide;
       }
       s_next += nsteps;
     }
     named_barrier(1, CSRB_HELPERS);  // the plan of the block is in shared memory
     const int nsteps = B.meta.nsteps, nent = B.meta.nent;
-    if (!B.meta.direct) {
+    if (!B.meta.direct && nsteps > 0) {
       // nonzeros of the block's rows: asynchronous 4-byte copies, all in flight together
       for (int r = warp - 1; r < nsteps; r += CSRB_HELPERS / 32) {
         const long long g0 = B.gbeg[r];
@@ -215,30 +275,124 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
         }
         B.slot[e] = (unsigned short)h;
       }
+      named_barrier(1, CSRB_HELPERS);  // the list of distinct columns is complete
+      // u at the block's columns (stale where the running block writes: see the boundary)
+      csrb_gather(B, cache, u, B.meta.nuniq, (int)threadIdx.x - 32, CSRB_HELPERS);
     }
   };
 
-  if (warp != 0) prepare(sm.buf[0]);
+  // ---- the steps of a block, chain warp, in shared memory ----------------------------------------------------------
+  auto run_steps = [&](CsrBlockBuf& B, float* cache, int nsteps, auto wide_tag) {
+    constexpr bool WIDE = decltype(wide_tag)::value;
+    float* red = sm.red;
+    int n_beg = B.rbeg[0], n_cnt = B.rcnt[0];
+    float n_y = B.yv[0], n_sb = B.sbef[0], n_eos = B.eos[0];
+    int n_sl[2];
+    float n_v[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int o = lane + 32 * q;
+      n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
+      n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
+    }
+    for (int r = 0; r < nsteps; ++r) {
+      const int beg = n_beg, cnt = n_cnt;
+      const float yy = n_y, sb = n_sb, eos = n_eos;
+      const int sl0 = n_sl[0], sl1 = n_sl[1];
+      const float v0 = n_v[0], v1 = n_v[1];
+      const bool in0 = lane < cnt, in1 = lane + 32 < cnt;
+      const float uq0 = in0 ? cache[sl0] : 0.0f;
+      const float uq1 = in1 ? cache[sl1] : 0.0f;
+      if (r + 1 < nsteps) {  // the next step's row does not depend on this step
+        n_beg = B.rbeg[r + 1];
+        n_cnt = B.rcnt[r + 1];
+        n_y = B.yv[r + 1];
+        n_sb = B.sbef[r + 1];
+        n_eos = B.eos[r + 1];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int o = lane + 32 * q;
+          n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
+          n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
+        }
+      }
+      float part = fmaf(uq1, v1, uq0 * v0);
+      if (WIDE)
+        for (int o = lane + 64; o < cnt; o += 32) part = fmaf(cache[B.slot[beg + o]], B.val[beg + o], part);
+      // sum over the warp through shared memory: every lane adds the 32 partial sums in the same order
+      red[lane] = part;
+      __syncwarp();
+      float4 a[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = ((const float4*)red)[i];
+      float t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = (a[i].x + a[i].y) + (a[i].z + a[i].w);
+      const float acc = ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + (t[6] + t[7]));
+      const float g = loss_derivative(LOSS, yy, sb * acc);
+      const float coef = eos * g;  // g == 0 (hinge off the margin): the stores below rewrite the same values
+      if (in0) cache[sl0] = fmaf(-coef, v0, uq0);
+      if (in1) cache[sl1] = fmaf(-coef, v1, uq1);
+      if (WIDE)
+        for (int o = lane + 64; o < cnt; o += 32) {
+          const int h = B.slot[beg + o];
+          cache[h] = fmaf(-coef, B.val[beg + o], cache[h]);
+        }
+      __syncwarp();  // the next step's slot loads see this step's stores; red can be written again
+    }
+  };
+
+  if (warp != 0) prepare(sm.buf[0], sm.ucache[0]);
   __syncthreads();
 
+  int prev_direct = 0;
   for (long long b = 0;; ++b) {
     CsrBlockBuf& B = sm.buf[b & 1];
-    const int nsteps = B.meta.nsteps;
-    if (nsteps == 0) break;
-    const int nuniq = B.meta.nuniq, direct = B.meta.direct;
+    CsrBlockBuf& Bp = sm.buf[(b + 1) & 1];  // the block that has just run (and the buffer of the next preparation)
+    float* cache = sm.ucache[b & 1];
+    float* cache_p = sm.ucache[(b + 1) & 1];
+    const int nsteps = B.meta.nsteps, nuniq = B.meta.nuniq, direct = B.meta.direct;
+    const int nuniq_p = Bp.meta.nuniq;
     const float fold = B.meta.fold;
-    if (fold != 0.0f) {  // rare: the scale was folded back before this block
-      for (long long c = threadIdx.x; c < p.d; c += CSRB_THREADS) u[c] = __ldcg(u + c) * fold;
+    const bool slow = b == 0 || nsteps == 0 || fold != 0.0f || direct || prev_direct;
+    if (!slow) {
+      // ---- boundary: columns that the block that has just run also holds take its values -----------------------------
+      for (int i = threadIdx.x; i < nuniq; i += CSRB_THREADS) {
+        const int h2 = B.uslot[i];
+        const int col = B.keys[h2];
+        int h = csrb_hash(col);
+        for (int probe = 0; probe < CSRB_HASH; ++probe) {
+          const int k2 = Bp.keys[h];
+          if (k2 == col) {
+            cache[h2] = cache_p[h];
+            break;
+          }
+          if (k2 == -1) break;
+          h = (h + 1) & (CSRB_HASH - 1);
+        }
+      }
+      __syncthreads();
+    } else {
+      // ---- slow boundary: write back, fold, read again ------------------------------------------------------------------
+      csrb_scatter(Bp, cache_p, u, nuniq_p, threadIdx.x, CSRB_THREADS);
+      __syncthreads();
+      if (threadIdx.x == 0) Bp.meta.nuniq = 0;
+      if (nsteps == 0) break;
+      if (fold != 0.0f) {
+        for (long long c = threadIdx.x; c < p.d; c += CSRB_THREADS) u[c] = __ldcg(u + c) * fold;
+        __syncthreads();
+      }
+      csrb_gather(B, cache, u, nuniq, threadIdx.x, CSRB_THREADS);
       __syncthreads();
     }
-    // ---- this block's columns of u into the cache (loads that bypass L1: other threads of the CTA wrote u) -------
-    for (int i = threadIdx.x; i < nuniq; i += CSRB_THREADS) {
-      const int h = B.uslot[i];
-      sm.ucache[h] = __ldcg(u + B.keys[h]);
-    }
-    __syncthreads();
     if (warp != 0) {
-      prepare(sm.buf[(b + 1) & 1]);
+      // the block that has just run goes back to u (a slow boundary has done it already: nothing left to do), then its
+      // tables and cache take the block after this one
+      csrb_scatter(Bp, cache_p, u, Bp.meta.nuniq, (int)threadIdx.x - 32, CSRB_HELPERS);
+      named_barrier(1, CSRB_HELPERS);
+      if (threadIdx.x == 32) Bp.meta.nuniq = 0;
+      named_barrier(1, CSRB_HELPERS);
+      prepare(Bp, cache_p);
     } else if (direct) {
       // ---- a single long row, on global memory ---------------------------------------------------------------
       const long long g0 = B.gbeg[0], g1 = B.gbeg[1];
@@ -257,70 +411,12 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
           if ((unsigned long long)(long long)c < (unsigned long long)p.d) u[c] = fmaf(-coef, p.val[o], __ldcg(u + c));
         }
       }
+    } else if (B.meta.wide) {
+      run_steps(B, cache, nsteps, std::true_type());
     } else {
-      // ---- the block's steps, in shared memory ------------------------------------------------------------------
-      constexpr int Q = 2;  // nonzeros per lane held in registers (rows of up to 64 nonzeros); longer rows loop
-      int n_beg = B.rbeg[0], n_cnt = B.rcnt[0];
-      float n_y = B.yv[0], n_sb = B.sbef[0], n_eos = B.eos[0];
-      int n_sl[Q];
-      float n_v[Q];
-#pragma unroll
-      for (int q = 0; q < Q; ++q) {
-        const int o = lane + 32 * q;
-        n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
-        n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
-      }
-      for (int r = 0; r < nsteps; ++r) {
-        const int beg = n_beg, cnt = n_cnt;
-        const float yy = n_y, sb = n_sb, eos = n_eos;
-        int sl[Q];
-        float v[Q], uq[Q];
-#pragma unroll
-        for (int q = 0; q < Q; ++q) {
-          sl[q] = n_sl[q];
-          v[q] = n_v[q];
-          uq[q] = sm.ucache[sl[q]];
-        }
-        if (r + 1 < nsteps) {  // the next step's row does not depend on this step
-          n_beg = B.rbeg[r + 1];
-          n_cnt = B.rcnt[r + 1];
-          n_y = B.yv[r + 1];
-          n_sb = B.sbef[r + 1];
-          n_eos = B.eos[r + 1];
-#pragma unroll
-          for (int q = 0; q < Q; ++q) {
-            const int o = lane + 32 * q;
-            n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
-            n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
-          }
-        }
-        float acc = 0.0f;
-#pragma unroll
-        for (int q = 0; q < Q; ++q) acc = fmaf(uq[q], v[q], acc);
-        for (int o = lane + 32 * Q; o < cnt; o += 32) acc = fmaf(sm.ucache[B.slot[beg + o]], B.val[beg + o], acc);
-        acc = warp_sum(acc);
-        const float g = loss_derivative(LOSS, yy, sb * acc);
-        if (g != 0.0f) {
-          const float coef = eos * g;
-#pragma unroll
-          for (int q = 0; q < Q; ++q)
-            if (lane + 32 * q < cnt) sm.ucache[sl[q]] = fmaf(-coef, v[q], uq[q]);
-          for (int o = lane + 32 * Q; o < cnt; o += 32) {
-            const int h = B.slot[beg + o];
-            sm.ucache[h] = fmaf(-coef, B.val[beg + o], sm.ucache[h]);
-          }
-        }
-        __syncwarp();  // the next step's slot loads must see this step's stores
-      }
+      run_steps(B, cache, nsteps, std::false_type());
     }
-    __syncthreads();
-    // ---- the block's slots back to u; its table is free again ----------------------------------------------------
-    for (int i = threadIdx.x; i < nuniq; i += CSRB_THREADS) {
-      const int h = B.uslot[i];
-      u[B.keys[h]] = sm.ucache[h];
-      B.keys[h] = -1;
-    }
-    if (threadIdx.x == 0) B.meta.nuniq = 0;
+    prev_direct = direct;
     __syncthreads();
   }
   if (warp == 1 && lane == 0) p.scale[j] = sc;
