@@ -12,7 +12,7 @@
 // distinct column among them a slot in a shared-memory hash table (linear probing, one compare-and-swap per
 // nonzero), store per nonzero its slot and value, and read u at the block's columns into the block's cache, all
 // while the chain warp runs the previous block. The chain warp runs a block's steps entirely in shared memory: slot
-// loads, a reduction over the warp through shared memory, the loss derivative, slot stores.
+// loads, a warp reduction, the loss derivative, slot stores.
 //
 // Block boundary. The values the helpers read for block b + 1 are stale exactly at the columns block b touches, so
 // at the boundary every column of block b + 1 is looked up in block b's table and, when found, takes block b's
@@ -62,10 +62,7 @@ struct CsrBlockBuf {
   unsigned short slot[CSRB_EMAX];      // slot of every nonzero
   unsigned short uslot[CSRB_EMAX];     // the occupied slots, in order of first insertion
   long long gbeg[CSRB_STEPS];          // first nonzero of the step's row in col_idx / val
-  int rbeg[CSRB_STEPS];                // first nonzero of the step within the block
-  int rcnt[CSRB_STEPS];                // nonzeros of the step's row
-  float yv[CSRB_STEPS];                // label
-  float sbef[CSRB_STEPS];              // scale before the step
+  int4 step[CSRB_STEPS];               // per step: first nonzero within the block, nonzeros, label bits, scale-before bits
   float eos[CSRB_STEPS];               // eta_n / scale after the step
   CsrBlockMeta meta;
 };
@@ -74,11 +71,48 @@ struct CsrBlockSmem {
   CsrBlockBuf buf[2];
   float ucache[2][CSRB_HASH];          // u at the columns of a block, by slot
   int colbuf[CSRB_EMAX];               // columns of the block being prepared
-  float red[32];                       // the chain warp's partial sums of a margin
 };
 
 __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Shared-memory accesses by 32-bit shared-window address. The block buffers are chosen at run time (b & 1), so the
+// hot loops name the state space themselves instead of leaving it to address-space inference.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ float lds_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ int lds_s32(uint32_t a) {
+  int v;
+  asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ int lds_u16(uint32_t a) {
+  unsigned short v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return (int)v;
+}
+__device__ __forceinline__ int4 lds_s32x4(uint32_t a) {
+  int4 v;
+  asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+__device__ __forceinline__ void sts_u16(uint32_t a, int v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"((unsigned short)v) : "memory");
+}
+__device__ __forceinline__ int atoms_cas(uint32_t a, int cmp, int val) {
+  int old;
+  asm volatile("atom.shared.cas.b32 %0, [%1], %2, %3;" : "=r"(old) : "r"(a), "r"(cmp), "r"(val) : "memory");
+  return old;
+}
+__device__ __forceinline__ int atoms_add(uint32_t a, int val) {
+  int old;
+  asm volatile("atom.shared.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(a), "r"(val) : "memory");
+  return old;
 }
 
 __device__ __forceinline__ int csrb_hash(int col) { return (int)(((uint32_t)col * 0x9E3779B1u) >> (32 - CSRB_HASH_BITS)); }
@@ -199,10 +233,7 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
         if (lane < n_ok) {
           const int r = nsteps + lane;
           B.gbeg[r] = gb[part];
-          B.rbeg[r] = nent + icnt - cnt;
-          B.rcnt[r] = cnt;
-          B.yv[r] = yy[part];
-          B.sbef[r] = (float)(sc * ea);
+          B.step[r] = make_int4(nent + icnt - cnt, cnt, __float_as_int(yy[part]), __float_as_int((float)(sc * ea)));
           B.eos[r] = (float)(eta / (sc * ia));
         }
         wide |= __any_sync(0xffffffffu, lane < n_ok && cnt > 64) ? 1 : 0;
@@ -212,10 +243,7 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
           if (lane == 0) {
             B.gbeg[0] = gb[part];
             B.gbeg[1] = ge[part];  // the row's end travels in the unused second entry
-            B.rbeg[0] = 0;
-            B.rcnt[0] = 0;
-            B.yv[0] = yy[part];
-            B.sbef[0] = (float)sc;
+            B.step[0] = make_int4(0, 0, __float_as_int(yy[part]), __float_as_int((float)sc));
             B.eos[0] = (float)(eta / (sc * a));
           }
           direct = 1;
@@ -247,7 +275,7 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
       // nonzeros of the block's rows: asynchronous 4-byte copies, all in flight together
       for (int r = warp - 1; r < nsteps; r += CSRB_HELPERS / 32) {
         const long long g0 = B.gbeg[r];
-        const int off = B.rbeg[r], cnt = B.rcnt[r];
+        const int off = B.step[r].x, cnt = B.step[r].y;
         for (int o = lane; o < cnt; o += 32) {
           cp_async4(&sm.colbuf[off + o], p.col_idx + g0 + o);
           cp_async4(&B.val[off + o], p.val + g0 + o);
@@ -256,24 +284,40 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
       cp_async_commit();
       cp_async_wait(0);
       named_barrier(1, CSRB_HELPERS);  // every helper's copies have landed
-      for (int e = (int)threadIdx.x - 32; e < nent; e += CSRB_HELPERS) {
-        int col = sm.colbuf[e];
-        if ((unsigned long long)(long long)col >= (unsigned long long)p.d) {
-          set_status(p.status, DEV_BOUNDS, 21, (long long)col);
-          col = 0;
-          B.val[e] = 0.0f;
-        }
-        int h = csrb_hash(col);
-        for (int probe = 0; probe < CSRB_HASH; ++probe) {
-          const int old = atomicCAS(&B.keys[h], -1, col);
-          if (old == -1) {
-            B.uslot[atomicAdd(&B.meta.nuniq, 1)] = (unsigned short)h;
-            break;
+      const uint32_t keys_a = smem_addr(B.keys), slot_a = smem_addr(B.slot), uslot_a = smem_addr(B.uslot);
+      const uint32_t col_a = smem_addr(sm.colbuf), nuniq_a = smem_addr(&B.meta.nuniq);
+      for (int e0 = 0; e0 < nent; e0 += CSRB_HELPERS) {  // the same trip count for every lane of a warp
+        const int e = e0 + (int)threadIdx.x - 32;
+        bool fresh = false;
+        int h = 0;
+        if (e < nent) {
+          int col = lds_s32(col_a + 4u * (uint32_t)e);
+          if ((unsigned long long)(long long)col >= (unsigned long long)p.d) {
+            set_status(p.status, DEV_BOUNDS, 21, (long long)col);
+            col = 0;
+            B.val[e] = 0.0f;
           }
-          if (old == col) break;
-          h = (h + 1) & (CSRB_HASH - 1);
+          h = csrb_hash(col);
+          for (int probe = 0; probe < CSRB_HASH; ++probe) {
+            const int old = atoms_cas(keys_a + 4u * (uint32_t)h, -1, col);
+            if (old == -1) {
+              fresh = true;
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(u + col));  // the block's read of u[col] follows soon
+              break;
+            }
+            if (old == col) break;
+            h = (h + 1) & (CSRB_HASH - 1);
+          }
+          sts_u16(slot_a + 2u * (uint32_t)e, h);
         }
-        B.slot[e] = (unsigned short)h;
+        // one counter update per warp for the columns seen for the first time
+        const unsigned fm = __ballot_sync(0xffffffffu, fresh);
+        if (fm) {
+          int base = 0;
+          if (lane == 0) base = atoms_add(nuniq_a, __popc(fm));
+          base = __shfl_sync(0xffffffffu, base, 0);
+          if (fresh) sts_u16(uslot_a + 2u * (uint32_t)(base + __popc(fm & ((1u << lane) - 1u))), h);
+        }
       }
       named_barrier(1, CSRB_HELPERS);  // the list of distinct columns is complete
       // u at the block's columns (stale where the running block writes: see the boundary)
@@ -284,61 +328,57 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
   // ---- the steps of a block, chain warp, in shared memory ----------------------------------------------------------
   auto run_steps = [&](CsrBlockBuf& B, float* cache, int nsteps, auto wide_tag) {
     constexpr bool WIDE = decltype(wide_tag)::value;
-    float* red = sm.red;
-    int n_beg = B.rbeg[0], n_cnt = B.rcnt[0];
-    float n_y = B.yv[0], n_sb = B.sbef[0], n_eos = B.eos[0];
-    int n_sl[2];
-    float n_v[2];
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const int o = lane + 32 * q;
-      n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
-      n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
+    const uint32_t cache_a = smem_addr(cache), step_a = smem_addr(B.step), eos_a = smem_addr(B.eos);
+    const uint32_t slot_a = smem_addr(B.slot) + 2u * (uint32_t)lane, val_a = smem_addr(B.val) + 4u * (uint32_t)lane;
+    // registers of the next step: its row does not depend on the running step
+    int4 n_st = lds_s32x4(step_a);
+    float n_eos = lds_f32(eos_a);
+    uint32_t n_c0 = cache_a, n_c1 = cache_a;  // addresses of the lane's two cached model entries
+    float n_v0 = 0.0f, n_v1 = 0.0f;
+    if (lane < n_st.y) {
+      n_c0 = cache_a + 4u * (uint32_t)lds_u16(slot_a + 2u * (uint32_t)n_st.x);
+      n_v0 = lds_f32(val_a + 4u * (uint32_t)n_st.x);
+    }
+    if (lane + 32 < n_st.y) {
+      n_c1 = cache_a + 4u * (uint32_t)lds_u16(slot_a + 2u * (uint32_t)(n_st.x + 32));
+      n_v1 = lds_f32(val_a + 4u * (uint32_t)(n_st.x + 32));
     }
     for (int r = 0; r < nsteps; ++r) {
-      const int beg = n_beg, cnt = n_cnt;
-      const float yy = n_y, sb = n_sb, eos = n_eos;
-      const int sl0 = n_sl[0], sl1 = n_sl[1];
-      const float v0 = n_v[0], v1 = n_v[1];
+      const int beg = n_st.x, cnt = n_st.y;
+      const float yy = __int_as_float(n_st.z), sb = __int_as_float(n_st.w), eos = n_eos;
+      const uint32_t c0 = n_c0, c1 = n_c1;
+      const float v0 = n_v0, v1 = n_v1;
       const bool in0 = lane < cnt, in1 = lane + 32 < cnt;
-      const float uq0 = in0 ? cache[sl0] : 0.0f;
-      const float uq1 = in1 ? cache[sl1] : 0.0f;
-      if (r + 1 < nsteps) {  // the next step's row does not depend on this step
-        n_beg = B.rbeg[r + 1];
-        n_cnt = B.rcnt[r + 1];
-        n_y = B.yv[r + 1];
-        n_sb = B.sbef[r + 1];
-        n_eos = B.eos[r + 1];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const int o = lane + 32 * q;
-          n_sl[q] = o < n_cnt ? B.slot[n_beg + o] : 0;
-          n_v[q] = o < n_cnt ? B.val[n_beg + o] : 0.0f;
+      float uq0 = 0.0f, uq1 = 0.0f;
+      if (in0) uq0 = lds_f32(c0);
+      if (in1) uq1 = lds_f32(c1);
+      if (r + 1 < nsteps) {
+        n_st = lds_s32x4(step_a + 16u * (uint32_t)(r + 1));
+        n_eos = lds_f32(eos_a + 4u * (uint32_t)(r + 1));
+        n_v0 = n_v1 = 0.0f;
+        if (lane < n_st.y) {
+          n_c0 = cache_a + 4u * (uint32_t)lds_u16(slot_a + 2u * (uint32_t)n_st.x);
+          n_v0 = lds_f32(val_a + 4u * (uint32_t)n_st.x);
+        }
+        if (lane + 32 < n_st.y) {
+          n_c1 = cache_a + 4u * (uint32_t)lds_u16(slot_a + 2u * (uint32_t)(n_st.x + 32));
+          n_v1 = lds_f32(val_a + 4u * (uint32_t)(n_st.x + 32));
         }
       }
       float part = fmaf(uq1, v1, uq0 * v0);
       if (WIDE)
         for (int o = lane + 64; o < cnt; o += 32) part = fmaf(cache[B.slot[beg + o]], B.val[beg + o], part);
-      // sum over the warp through shared memory: every lane adds the 32 partial sums in the same order
-      red[lane] = part;
-      __syncwarp();
-      float4 a[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) a[i] = ((const float4*)red)[i];
-      float t[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) t[i] = (a[i].x + a[i].y) + (a[i].z + a[i].w);
-      const float acc = ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + (t[6] + t[7]));
+      const float acc = warp_sum(part);  // shuffles only: nothing here waits on shared memory
       const float g = loss_derivative(LOSS, yy, sb * acc);
       const float coef = eos * g;  // g == 0 (hinge off the margin): the stores below rewrite the same values
-      if (in0) cache[sl0] = fmaf(-coef, v0, uq0);
-      if (in1) cache[sl1] = fmaf(-coef, v1, uq1);
+      if (in0) sts_f32(c0, fmaf(-coef, v0, uq0));
+      if (in1) sts_f32(c1, fmaf(-coef, v1, uq1));
       if (WIDE)
         for (int o = lane + 64; o < cnt; o += 32) {
           const int h = B.slot[beg + o];
           cache[h] = fmaf(-coef, B.val[beg + o], cache[h]);
         }
-      __syncwarp();  // the next step's slot loads see this step's stores; red can be written again
+      __syncwarp();  // the next step's slot loads see this step's stores
     }
   };
 
@@ -357,14 +397,16 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
     const bool slow = b == 0 || nsteps == 0 || fold != 0.0f || direct || prev_direct;
     if (!slow) {
       // ---- boundary: columns that the block that has just run also holds take its values -----------------------------
+      const uint32_t uslot_a = smem_addr(B.uslot), keys_a = smem_addr(B.keys), keysp_a = smem_addr(Bp.keys);
+      const uint32_t cache_a = smem_addr(cache), cachep_a = smem_addr(cache_p);
       for (int i = threadIdx.x; i < nuniq; i += CSRB_THREADS) {
-        const int h2 = B.uslot[i];
-        const int col = B.keys[h2];
+        const int h2 = lds_u16(uslot_a + 2u * (uint32_t)i);
+        const int col = lds_s32(keys_a + 4u * (uint32_t)h2);
         int h = csrb_hash(col);
         for (int probe = 0; probe < CSRB_HASH; ++probe) {
-          const int k2 = Bp.keys[h];
+          const int k2 = lds_s32(keysp_a + 4u * (uint32_t)h);
           if (k2 == col) {
-            cache[h2] = cache_p[h];
+            sts_f32(cache_a + 4u * (uint32_t)h2, lds_f32(cachep_a + 4u * (uint32_t)h));
             break;
           }
           if (k2 == -1) break;
@@ -403,7 +445,7 @@ __global__ void __launch_bounds__(CSRB_THREADS, 1) chain_csr_block_kernel(const 
         else set_status(p.status, DEV_BOUNDS, 22, (long long)c);
       }
       acc = warp_sum(acc);
-      const float g = loss_derivative(LOSS, B.yv[0], B.sbef[0] * acc);
+      const float g = loss_derivative(LOSS, __int_as_float(B.step[0].z), __int_as_float(B.step[0].w) * acc);
       if (g != 0.0f) {
         const float coef = B.eos[0] * g;
         for (long long o = g0 + lane; o < g1; o += 32) {
