@@ -4,14 +4,17 @@ Some users of the library run where cudaMalloc is off limits: inside a framework
 already owns the device, in a loop that cannot take cudaMalloc's device-wide synchronisation, or
 in a process with a memory budget fixed at start-up. For them the library carries its working
 memory (models, sample stream, tables) in an array compiled into it. This test calls that entry point
-through the C ABI and compares it with the ordinary context-based path on the same inputs, twice in
-a row with different problem sizes, because all calls share the one array and the second call meets
-the first call's leftovers. The file is named so that pytest collects it last.
+through the C ABI and compares it with the ordinary context-based path and with the CPU oracle on the
+same inputs, several times in a row with different problem sizes, because all calls share the one array
+and every call meets the previous call's leftovers. It also checks the two promises such a caller
+relies on: the library takes no device memory during the calls, and a problem inside the kernels is
+reported through wpsgd_check_static. The file is named so that pytest collects it last.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import wpsgd_inputs as wi
 
 pytestmark = pytest.mark.gpu
@@ -32,22 +35,48 @@ def _context_path(P, wl, r):
     return v
 
 
-def test_no_alloc_entry_point_matches_context_path_twice_in_a_row(wpsgd_lib):
+def _cases():
+    first = wi.config2(k=6, d=512, m=128, base_steps=400)      # larger problem first ...
+    first.w0 = torch.full((512,), 0.25)
+    second = wi.config1(k=3, d=64, m=64, n_steps=(90, 0, 31))  # ... then a smaller one over its leftovers
+    third = wi.config3(k=4, d=1024, m=64, n_lo=50, n_hi=300)   # bf16 rows
+    return [(first, 0.0), (second, 0.999), (third, 0.0), (first, 0.0)]
+
+
+def test_no_alloc_entry_point_matches_context_path_and_oracle_calls_in_a_row(wpsgd_lib):
     import paper_1708_04801_b200 as P
 
-    first = wi.config2(k=6, d=512, m=128, base_steps=400).to("cuda")      # larger problem first ...
-    first.w0 = torch.full((512,), 0.25, device="cuda")
-    second = wi.config1(k=3, d=64, m=64, n_steps=(90, 0, 31)).to("cuda")  # ... then a smaller one over its leftovers
-    third = wi.config3(k=4, d=1024, m=64, n_lo=50, n_hi=300).to("cuda")   # bf16 rows
-    for wl, r in ((first, 0.0), (second, 0.999), (third, 0.0), (first, 0.0)):
+    for wl_cpu, r in _cases():
+        wl = wl_cpu.to("cuda")
         out = torch.full((wl.d,), float("nan"), dtype=torch.float32, device="cuda")  # caller-owned output
         P.solve_static(wl.X, wl.y, wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed, w0=wl.w0,
                        r=r, out=out)
-        torch.cuda.synchronize()
+        P.check_static(0)  # waits for the stream; raises if a kernel flagged a timeout or a bounds failure
         got = out.cpu().numpy()
-        want = _context_path(P, wl, r)
         assert np.isfinite(got).all()
+        assert _rel_l2(got, _context_path(P, wl, r)) <= TOL[wl.loss]
+        want, _, _ = oracle.solve(wl_cpu, r)  # the CPU checker shares no code with either CUDA path
         assert _rel_l2(got, want) <= TOL[wl.loss]
+
+
+def test_no_alloc_entry_point_takes_no_device_memory(wpsgd_lib):
+    import paper_1708_04801_b200 as P
+
+    cases = [(wl.to("cuda"), r) for wl, r in _cases()]
+    outs = [torch.empty(wl.d, dtype=torch.float32, device="cuda") for wl, _ in cases]
+    wl, r = cases[0]
+    P.solve_static(wl.X, wl.y, wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed, w0=wl.w0, r=r,
+                   out=outs[0])  # first call on the device: module load and the look-up of the array's address
+    P.check_static(0)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for (wl, r), out in zip(cases, outs):
+        P.solve_static(wl.X, wl.y, wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed, w0=wl.w0, r=r,
+                       out=out)
+        P.check_static(0)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "wpsgd_solve_static or wpsgd_check_static changed the free device memory"
 
 
 def test_no_alloc_entry_point_rejects_sizes_beyond_its_array(wpsgd_lib):
