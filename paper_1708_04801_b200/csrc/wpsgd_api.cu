@@ -14,6 +14,7 @@
 #include "chain_csr.cuh"
 #include "chain_csr_block.cuh"
 #include "chain_mma.cuh"
+#include "chain_mma16.cuh"
 #include "chain_dense.cuh"
 #include "combine.cuh"
 #include "philox.cuh"
@@ -63,6 +64,7 @@ struct wpsgd_ctx {
   // options
   int opt_stages = 0;
   int opt_variant = 0, opt_prefetch = 0, opt_threads = 0, opt_cluster = 0;
+  int opt_block_samples = 0;   // tensor-core cluster kernel: samples per block (0: chosen here, 8 or 16)
   int opt_sparse_variant = 0;  // 0: chosen here, 1: one step per round trip, 2: blocks of steps through a shared-memory cache
   long long opt_spin_limit = 1ll << 20;
   long long opt_drop_block = -1;
@@ -380,6 +382,8 @@ wpsgd_status launch_block(wpsgd_ctx* c, const ChainParams& p, int threads, int R
 // ---- bf16 rows: Gram block and margins on the tensor cores, columns split over a cluster -------------------------------
 struct ClusterShape {
   int C = 1, cpc = 0, math_warps = 1, stages = 2;
+  int block = 8;    // samples per block
+  int stages16 = 0; // ring depth of the 16-sample form (0: it does not fit)
 };
 
 bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
@@ -417,6 +421,13 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   out->cpc = (int)cpc;
   out->math_warps = (int)mw;
   out->stages = stages;
+  // 16 samples per block (squared and hinge losses): half as many hand-offs per sample; one CTA per SM
+  int s16 = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
+  while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16).total > kSmemBudget) --s16;
+  out->stages16 = s16 >= 2 ? s16 : 0;
+  const bool can16 = out->stages16 > 0 && c->loss != WPSGD_LOSS_LOGISTIC;
+  out->block = (c->opt_block_samples == 16 || (c->opt_block_samples == 0 && can16)) ? 16 : 8;
+  if (out->block == 16 && !can16) return false;
   return true;
 }
 
@@ -429,7 +440,9 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   cp.b.drop_block = c->opt_drop_block;
   cp.b.group_order = nullptr;
   cp.chunks_per_cta = sh.cpc;
-  const size_t smem = MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
+  const bool b16 = sh.block == 16;
+  if (b16) cp.b.stages = sh.stages16;
+  const size_t smem = b16 ? Mma16Smem(sh.stages16, (size_t)sh.cpc * 16).total : MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
@@ -448,6 +461,7 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
     c->launches++;
     return WPSGD_OK;
   };
+  if (b16) return c->loss == WPSGD_LOSS_HINGE ? go(chain_mma16_kernel<LOSS_HINGE>) : go(chain_mma16_kernel<LOSS_SQUARED>);
   switch (c->loss) {
     case WPSGD_LOSS_HINGE: return go(chain_mma_kernel<LOSS_HINGE, 4>);
     case WPSGD_LOSS_LOGISTIC: return go(chain_mma_kernel<LOSS_LOGISTIC, 4>);
@@ -852,6 +866,9 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   } else if (n == "host_pipeline") {
     if (value != 0 && value != 1) return fail(c, WPSGD_ERR_INVALID_ARG, "host_pipeline must be 0 or 1");
     c->opt_host_pipeline = (int)value;
+  } else if (n == "block_samples") {
+    if (value != 0 && value != 8 && value != 16) return fail(c, WPSGD_ERR_INVALID_ARG, "block_samples must be 0, 8 or 16");
+    c->opt_block_samples = (int)value;
   } else if (n == "sparse_variant") {
     if (value < 0 || value > 2) return fail(c, WPSGD_ERR_INVALID_ARG, "sparse_variant must be 0, 1 or 2");
     c->opt_sparse_variant = (int)value;

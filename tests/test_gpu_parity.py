@@ -229,14 +229,23 @@ def test_bounded_wait_for_rows_reports_timeout_and_context_survives(P, d, bf16):
     assert rel_l2(v, ov) <= 1e-4
 
 
-# ---- tensor-core cluster kernel (bf16 rows): Gram block and margins from mma, model split into three bf16 rows ----------
-TC_VARIANTS = [8]
+# ---- tensor-core cluster kernel (bf16 rows): Gram block and margins from mma, model split into three bf16 rows; blocks
+# of 8 samples (every loss) or 16 samples (squared and hinge) -----------------------------------------------------------
+MMA_BLOCKS = [8, 16]
+
+
+def _mma(block, wl, **more):
+    """Options that select the tensor-core kernel with the given block size; the 16-sample form has no logistic loss."""
+    if block == 16 and wl.loss == LOGISTIC:
+        wl.loss = SQUARED
+        wl.y = (wl.y * 0.3).contiguous()
+    return dict({"dense_variant": 8, "block_samples": block}, **more)
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 4])
 @pytest.mark.parametrize("d", [480, 488, 8, 264])
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_ragged_shapes(P, cluster, d, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_ragged_shapes(P, cluster, d, block):
     # 60 / 61 / 1 / 33 chunks of 8 columns: odd chunk counts leave half a 16-column tile empty, the last CTA of a
     # cluster owns a ragged slice, and with d = 8 only one CTA can exist
     if d == 8 and cluster > 1:
@@ -245,48 +254,51 @@ def test_mma_kernel_ragged_shapes(P, cluster, d, variant):
     wl.n_steps[2] = 0
     wl.w0 = torch.full((d,), 0.05)
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": variant, "cluster": cluster})
+    assert_parity(P, wl, _mma(block, wl, cluster=cluster))
 
 
 @pytest.mark.parametrize("d,cluster", [(4096, 2), (4096, 4), (2048, 1), (4096, 8), (3008, 2), (1024, 8)])
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_losses_and_widths(P, d, cluster, loss, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_losses_and_widths(P, d, cluster, loss, block):
     wl = wi.config2(k=3, d=d, m=48, base_steps=210)
     wl.loss = loss
     if loss == SQUARED:
         wl.y = (wl.y * 0.3).contiguous()
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": variant, "cluster": cluster})
+    if block == 16 and loss == LOGISTIC:
+        pytest.skip("the 16-sample form has squared and hinge losses only")
+    assert_parity(P, wl, _mma(block, wl, cluster=cluster))
 
 
-@pytest.mark.parametrize("n_steps", [(1, 7, 8), (9, 15, 16), (17, 0, 64), (333, 250, 3)])
+@pytest.mark.parametrize("n_steps", [(1, 7, 8), (9, 15, 16), (17, 0, 64), (333, 250, 3), (31, 32, 33)])
 @pytest.mark.parametrize("stages", [2, 3, 4])
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_block_boundaries_and_ring_depths(P, n_steps, stages, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_block_boundaries_and_ring_depths(P, n_steps, stages, block):
     wl = wi.config2(k=3, d=1024, m=64, base_steps=8)
     wl.n_steps = np.array(n_steps, dtype=np.int64)
     wl.w0 = torch.full((1024,), 0.1)
     wl.X = wl.X.to(torch.bfloat16)
-    assert_parity(P, wl, {"dense_variant": variant, "cluster": 2, "stages": stages})
+    assert_parity(P, wl, _mma(block, wl, cluster=2, stages=stages))
 
 
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_model_split_keeps_fp32_accuracy(P, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_model_split_keeps_fp32_accuracy(P, block):
     # a model with a wide spread of magnitudes (w0 from 1e-6 to 1e3): the three bf16 rows must carry all 24 bits of
     # every entry, or the margins of the first steps are off by far more than the tolerance
     wl = wi.config3(k=4, d=2048, m=64, n_lo=40, n_hi=90)
     g = torch.Generator().manual_seed(11)
     wl.w0 = (torch.randn(2048, generator=g) * torch.logspace(-6, 3, 2048)).contiguous()
-    assert_parity(P, wl, {"dense_variant": variant, "cluster": 2})
+    assert_parity(P, wl, _mma(block, wl, cluster=2))
 
 
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_default_shape_and_continue(P, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_default_shape_and_continue(P, block):
     wl_cpu = wi.small(3)
     wl = wl_cpu.to("cuda")
     with P.Context(wl.k, wl.d) as ctx:
-        ctx.set_option("dense_variant", variant)
+        ctx.set_option("dense_variant", 8)
+        ctx.set_option("block_samples", block)
         first = np.minimum(wl.n_steps, 301)
         ctx.run(wl.X, wl.y, wl.shard_off, first, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
         ctx.continue_(wl.X, wl.y, wl.shard_off, wl.n_steps - first)
@@ -297,29 +309,35 @@ def test_mma_kernel_default_shape_and_continue(P, variant):
         assert rel_l2(seg[j], oW[j]) <= 1e-4
 
 
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_limits(P, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_limits(P, block):
     wl = wi.config2(k=2, d=64, m=16, base_steps=20)  # fp32 rows
     with pytest.raises(P.WpsgdError) as e:
-        gpu_solve(P, wl, {"dense_variant": variant})
+        gpu_solve(P, wl, {"dense_variant": 8, "block_samples": block})
     assert e.value.status_name == "UNSUPPORTED"
     wl.X = wl.X.to(torch.bfloat16)  # 8 chunks: a cluster of 8 needs 8 non-empty slices; 16 CTAs cannot exist
     with pytest.raises(P.WpsgdError) as e:
-        gpu_solve(P, wl, {"dense_variant": variant, "cluster": 16})
+        gpu_solve(P, wl, {"dense_variant": 8, "block_samples": block, "cluster": 16})
     assert e.value.status_name == "INVALID_ARG"
+    if block == 16:  # logistic loss: the 16-sample form is refused, the default falls back to 8 samples
+        with pytest.raises(P.WpsgdError) as e:
+            gpu_solve(P, wl, {"dense_variant": 8, "block_samples": 16})
+        assert e.value.status_name == "UNSUPPORTED"
+        assert_parity(P, wl, {"dense_variant": 8})
 
 
 @pytest.mark.parametrize("d,cluster", [(1024, 1), (4096, 2), (4096, 4)])
-@pytest.mark.parametrize("variant", TC_VARIANTS)
-def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, cluster, variant):
+@pytest.mark.parametrize("block", MMA_BLOCKS)
+def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, cluster, block):
     # Failure detection without a fault: the rows of block 3 are never requested (test hook), so the bounded wait
     # for them runs out; every CTA of the cluster is told, all leave in step, and the next run is clean.
     wl_cpu = wi.config2(k=3, d=d, m=32, base_steps=120)
     wl_cpu.X = wl_cpu.X.to(torch.bfloat16)
+    opts = _mma(block, wl_cpu, cluster=cluster)
     wl = wl_cpu.to("cuda")
     with P.Context(wl.k, wl.d) as ctx:
-        ctx.set_option("dense_variant", variant)
-        ctx.set_option("cluster", cluster)
+        for k_, v_ in opts.items():
+            ctx.set_option(k_, v_)
         ctx.set_option("spin_limit", 2000)
         ctx.set_option("test_drop_block", 3)
         ctx.run_workload(wl)
