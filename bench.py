@@ -44,7 +44,12 @@ N_SMS = 148
 
 # DRAM bytes (read + write) per launch of the chain kernel from an ncu capture, with the hash of the
 # kernel sources the capture was taken from; reported as null once the sources have changed.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    "config3": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 26349015040,
+                "note": "captured with 2048 rows per node (2 GiB on the device): same step counts and kernel work per launch, no scaling"},
+    "config5": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 15945717400, "note": "full-size capture"},
+    "config4": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 4275997808, "note": "full-size capture"},
+}
 
 
 def parse_args():
