@@ -225,6 +225,86 @@ constexpr int BLK_B = 8;                           // samples per block
 constexpr int BLK_PAIRS = BLK_B * (BLK_B - 1) / 2;  // 28 Gram entries below the diagonal
 constexpr int BLK_MAX_MATH_WARPS = 16;
 
+// Per-sample constants of a block of 8 with everything folded in that does not depend on the chain:
+// t_n = sc_n (p_n - sum_m beta_m G_mn) is the argument of the loss derivative, beta_n = cf_n * f(t_n).
+// apw[m] = a^m, cfac[m] = eta / a^{m+1}; samples from nv on lie beyond the chain's end and take no step.
+template <int LOSS>
+__device__ __forceinline__ void block8_constants(const float (&yv)[BLK_B], const float (&apw)[BLK_B], const float (&cfac)[BLK_B],
+                                                 int nv, float (&sc)[BLK_B], float (&cf)[BLK_B]) {
+#pragma unroll
+  for (int m = 0; m < BLK_B; ++m) {
+    if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
+      sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
+      cf[m] = -yv[m] * cfac[m];
+    } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
+      sc[m] = yv[m] * apw[m];
+      cf[m] = -yv[m] * cfac[m];
+    } else {  // g = t - y, t = a^n (...)
+      sc[m] = apw[m];
+      cf[m] = cfac[m];
+    }
+    if (m >= nv) cf[m] = 0.0f;
+  }
+}
+
+// The 8-step scalar recurrence of a block, every lane the same (no shuffle in the dependent chain). On entry
+// t[n] = sc_n p_n and Gs[n (n - 1) / 2 + m] = sc_n G_mn (m < n); on exit beta[m] = eta g_m / a^{m+1}. For the logistic
+// loss jets_smem (8 float4 of the warp's own) receives the expansions of the factor around the block's margins:
+// lane n < 8 expands its own sample at t_own, every lane then reads all eight; a block whose steps move a margin
+// beyond the range of the cubic is run again with the direct evaluation.
+template <int LOSS>
+__device__ __forceinline__ void block8_recurrence(float (&t)[BLK_B], const float (&Gs)[BLK_PAIRS], const float (&cf)[BLK_B],
+                                                  const float (&yv)[BLK_B], float t_own, float4* jets_smem,
+                                                  float (&beta)[BLK_B]) {
+  constexpr int B = BLK_B;
+  if (LOSS == LOSS_LOGISTIC) {
+    const int lane = threadIdx.x & 31;
+    if (lane < B) jets_smem[lane] = logistic_jet(t_own);
+    __syncwarp();
+    float4 jet[B];
+    float dlt[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m) {
+      jet[m] = jets_smem[m];
+      dlt[m] = 0.0f;
+    }
+    float dmax = 0.0f;  // (jets_smem is written again a block later, behind at least one warp-wide barrier of the caller)
+#pragma unroll
+    for (int m = 0; m < B; ++m) {
+      dmax = fmaxf(dmax, fabsf(dlt[m]));
+      beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
+#pragma unroll
+      for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
+    }
+    if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
+#pragma unroll 1
+      for (int m = 0; m < B; ++m) {
+        float tm_ = 0.0f, cfm = 0.0f;
+#pragma unroll
+        for (int q = 0; q < B; ++q)
+          if (q == m) { tm_ = t[q]; cfm = cf[q]; }
+        const float bm = cfm * logistic_factor(tm_);
+#pragma unroll
+        for (int q = 0; q < B; ++q)
+          if (q == m) beta[q] = bm;
+#pragma unroll
+        for (int n2 = 1; n2 < B; ++n2)
+#pragma unroll
+          for (int q = 0; q < n2; ++q)
+            if (q == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + q], t[n2]);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int m = 0; m < B; ++m) {
+      if (LOSS == LOSS_HINGE) beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
+      else beta[m] = cf[m] * (t[m] - yv[m]);
+#pragma unroll
+      for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
+    }
+  }
+}
+
 // Shared-memory carve-up (bytes). Ring first (16-byte aligned), then the small arrays.
 struct BlockSmem {
   size_t ring, redG, redP, totG, gam, tab, jet, bars, flag, total;
@@ -316,24 +396,10 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       if (b + 1 < nb) y_nxt = yshard[id_nxt];
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
       const float a_nv = tab[nv], dl_nv = tab[32 + nv];
-      // per-sample constants with everything folded in that does not depend on the chain:
-      // t_n = sc_n (p_n - sum_m beta_m G_mn) is the argument of the loss derivative, beta_n = cf_n * f(t_n)
       float yv[B], sc[B], cf[B];
 #pragma unroll
-      for (int m = 0; m < B; ++m) {
-        yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
-        if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
-          sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
-          cf[m] = -yv[m] * cfac[m];
-        } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
-          sc[m] = yv[m] * apw[m];
-          cf[m] = -yv[m] * cfac[m];
-        } else {  // g = t - y, t = a^n (...)
-          sc[m] = apw[m];
-          cf[m] = cfac[m];
-        }
-        if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
-      }
+      for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+      block8_constants<LOSS>(yv, apw, cfac, nv, sc, cf);
       float Gs[BLK_PAIRS];  // sc_n G_mn at [n(n-1)/2 + m], m < n
       auto gather_gram = [&]() {
         {
@@ -376,55 +442,7 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
-      if (LOSS == LOSS_LOGISTIC) {
-        // lane n & 7 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
-        if (lane < B) jets[lane] = logistic_jet(y_cur * tab[n] * 1.4426950408889634f * psum);
-        __syncwarp();
-        float4 jet[B];
-        float dlt[B];
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          jet[m] = jets[m];
-          dlt[m] = 0.0f;
-        }
-        float dmax = 0.0f;
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          dmax = fmaxf(dmax, fabsf(dlt[m]));
-          beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
-#pragma unroll
-          for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
-        }
-        if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
-#pragma unroll 1
-          for (int m = 0; m < B; ++m) {
-            float tm_ = 0.0f, cfm = 0.0f;
-#pragma unroll
-            for (int q = 0; q < B; ++q)
-              if (q == m) { tm_ = t[q]; cfm = cf[q]; }
-            const float bm = cfm * logistic_factor(tm_);
-#pragma unroll
-            for (int q = 0; q < B; ++q)
-              if (q == m) beta[q] = bm;
-#pragma unroll
-            for (int n2 = 1; n2 < B; ++n2)
-#pragma unroll
-              for (int q = 0; q < n2; ++q)
-                if (q == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + q], t[n2]);
-          }
-        }
-      } else {
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          if (LOSS == LOSS_HINGE) {
-            beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
-          } else {
-            beta[m] = cf[m] * (t[m] - yv[m]);
-          }
-#pragma unroll
-          for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
-        }
-      }
+      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * psum, jets, beta);
       // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}
       float mine = dl_nv;
 #pragma unroll
@@ -686,7 +704,7 @@ struct BlockWarpSmem {
   __host__ __device__ BlockWarpSmem(int stages, size_t row_bytes, int warps) {
     ring = 0;
     scratch = ring + (size_t)warps * stages * BLK_B * row_bytes;
-    tab = scratch + (size_t)warps * 48 * sizeof(float);
+    tab = scratch + (size_t)warps * 72 * sizeof(float);
     total = tab + 3 * 16 * sizeof(float);
   }
 };
@@ -706,7 +724,7 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
   const int nwarps = blockDim.x >> 5;
   const BlockWarpSmem L(S, row_bytes, nwarps);
   unsigned char* ring = smem + L.ring + (size_t)warp * S * B * row_bytes;
-  float* scratch = (float*)(smem + L.scratch) + warp * 48;  // [0..27] G entries, [32..39] p
+  float* scratch = (float*)(smem + L.scratch) + warp * 72;  // [0..27] G entries, [32..39] p, [40..71] logistic expansions
   float* tab = (float*)(smem + L.tab);
 
   if (threadIdx.x <= B) {  // power tables in fp64, rounded once
@@ -852,75 +870,22 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
       const float4 q0 = ((const float4*)scratch)[8], q1 = ((const float4*)scratch)[9];
       pv[0] = q0.x; pv[1] = q0.y; pv[2] = q0.z; pv[3] = q0.w; pv[4] = q1.x; pv[5] = q1.y; pv[6] = q1.z; pv[7] = q1.w;
     }
+    const float pv_own = scratch[32 + n];  // margin of the sample this lane looks after
     __syncwarp();
     // ---- 8-step recurrence, every lane the same ----------------------------------------------------------
     const float a_nv = tab[nv], dl = tab[32 + nv];
-    float t[B], beta[B], yv[B], cf[B];
+    float t[B], beta[B], yv[B], cf[B], sc[B];
+#pragma unroll
+    for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+    block8_constants<LOSS>(yv, apw, cfac, nv, sc, cf);
 #pragma unroll
     for (int m = 0; m < B; ++m) {
-      yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
-      float sc;
-      if (LOSS == LOSS_LOGISTIC) { sc = yv[m] * apw[m] * 1.4426950408889634f; cf[m] = -yv[m] * cfac[m]; }
-      else if (LOSS == LOSS_HINGE) { sc = yv[m] * apw[m]; cf[m] = -yv[m] * cfac[m]; }
-      else { sc = apw[m]; cf[m] = cfac[m]; }
-      if (m >= nv) cf[m] = 0.0f;
-      t[m] = sc * pv[m];
+      t[m] = sc[m] * pv[m];
 #pragma unroll
-      for (int k2 = 0; k2 < m; ++k2) Gs[m * (m - 1) / 2 + k2] *= sc;
+      for (int k2 = 0; k2 < m; ++k2) Gs[m * (m - 1) / 2 + k2] *= sc[m];
     }
-    if (LOSS == LOSS_LOGISTIC) {
-      // lane n & 7 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
-      // through the warp's scratch line (its Gram entries and p are in registers by now)
-      const float t_own = y_cur * tab[n] * 1.4426950408889634f * scratch[32 + n];
-      __syncwarp();
-      if (lane < B) ((float4*)scratch)[lane] = logistic_jet(t_own);
-      __syncwarp();
-      float4 jet[B];
-      float dlt[B];
-#pragma unroll
-      for (int m = 0; m < B; ++m) {
-        jet[m] = ((const float4*)scratch)[m];
-        dlt[m] = 0.0f;
-      }
-      __syncwarp();
-      float dmax = 0.0f;
-#pragma unroll
-      for (int m = 0; m < B; ++m) {
-        dmax = fmaxf(dmax, fabsf(dlt[m]));
-        beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
-#pragma unroll
-        for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
-      }
-      if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
-#pragma unroll 1
-        for (int m = 0; m < B; ++m) {
-          float tm_ = 0.0f, cfm = 0.0f;
-#pragma unroll
-          for (int q = 0; q < B; ++q)
-            if (q == m) { tm_ = t[q]; cfm = cf[q]; }
-          const float bm = cfm * logistic_factor(tm_);
-#pragma unroll
-          for (int q = 0; q < B; ++q)
-            if (q == m) beta[q] = bm;
-#pragma unroll
-          for (int n2 = 1; n2 < B; ++n2)
-#pragma unroll
-            for (int q = 0; q < n2; ++q)
-              if (q == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + q], t[n2]);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int m = 0; m < B; ++m) {
-        if (LOSS == LOSS_HINGE) {
-          beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
-        } else {
-          beta[m] = cf[m] * (t[m] - yv[m]);
-        }
-#pragma unroll
-        for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
-      }
-    }
+    // lane n & 7 expands the logistic factor of its own sample around t0_n (scratch[40..71] holds the expansions)
+    block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * pv_own, (float4*)(scratch + 40), beta);
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m,  gamma_m = beta_m a^nv ----------------------------------
     {
       constexpr int NP = XPairs<XT>::NP;

@@ -212,20 +212,8 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
       const float a_nv = tab[nv], dl_nv = tab[32 + nv];
       float yv[B], sc[B], cf[B];
 #pragma unroll
-      for (int m = 0; m < B; ++m) {
-        yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
-        if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
-          sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
-          cf[m] = -yv[m] * cfac[m];
-        } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
-          sc[m] = yv[m] * apw[m];
-          cf[m] = -yv[m] * cfac[m];
-        } else {  // g = t - y, t = a^n (...)
-          sc[m] = apw[m];
-          cf[m] = cfac[m];
-        }
-        if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
-      }
+      for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
+      block8_constants<LOSS>(yv, apw, cfac, nv, sc, cf);
       // ---- wait (bounded) for the partial sums of block b from every math warp of the cluster ------------------
       {
         const uint32_t parity = (uint32_t)((b >> 1) & 1);
@@ -273,55 +261,7 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
-      if (LOSS == LOSS_LOGISTIC) {
-        // lane n < 8 expands the factor of its own sample around t0_n; every lane then fetches all eight expansions
-        if (lane < B) jets[lane] = logistic_jet(y_cur * tab[n] * 1.4426950408889634f * psum);
-        __syncwarp();
-        float4 jet[B];
-        float dlt[B];
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          jet[m] = jets[m];
-          dlt[m] = 0.0f;
-        }
-        float dmax = 0.0f;
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          dmax = fmaxf(dmax, fabsf(dlt[m]));
-          beta[m] = cf[m] * logistic_factor_near(jet[m], dlt[m]);
-#pragma unroll
-          for (int n2 = m + 1; n2 < B; ++n2) dlt[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], dlt[n2]);
-        }
-        if (!(dmax < LOGISTIC_DELTA_MAX)) {  // rare: some step of the block moved a margin far; direct evaluation
-#pragma unroll 1
-          for (int m = 0; m < B; ++m) {
-            float tm_ = 0.0f, cfm = 0.0f;
-#pragma unroll
-            for (int k = 0; k < B; ++k)
-              if (k == m) { tm_ = t[k]; cfm = cf[k]; }
-            const float bm = cfm * logistic_factor(tm_);
-#pragma unroll
-            for (int k = 0; k < B; ++k)
-              if (k == m) beta[k] = bm;
-#pragma unroll
-            for (int n2 = 1; n2 < B; ++n2)
-#pragma unroll
-              for (int k = 0; k < n2; ++k)
-                if (k == m) t[n2] = fmaf(-bm, Gs[n2 * (n2 - 1) / 2 + k], t[n2]);
-          }
-        }
-      } else {
-#pragma unroll
-        for (int m = 0; m < B; ++m) {
-          if (LOSS == LOSS_HINGE) {
-            beta[m] = (t[m] < 1.0f) ? cf[m] : 0.0f;
-          } else {
-            beta[m] = cf[m] * (t[m] - yv[m]);
-          }
-#pragma unroll
-          for (int n2 = m + 1; n2 < B; ++n2) t[n2] = fmaf(-beta[m], Gs[n2 * (n2 - 1) / 2 + m], t[n2]);
-        }
-      }
+      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * psum, jets, beta);
       // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}; [8] = 1 - a^nv; [9] = leave after this block
       float mine = dl_nv;
 #pragma unroll
