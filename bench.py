@@ -361,6 +361,9 @@ def measure(P, multi, wl, cfg, dev, steps, warmup, peak, peak_src, options, worl
             "ctas": ctas, "sm_coverage": min(1.0, ctas / N_SMS),
             # the serial side of the same kernel: device cycles per sample-update of the longest chain
             "cycles_per_update_longest_chain": chain_med * 1e-3 * mhz * 1e6 / max(longest, 1)}
+    # which side of the kernel holds it back: the memory system, or the dependent steps of one chain
+    roof["limiter"] = ("chain latency: the longest chain's dependent steps, not a memory level"
+                       if (roof["frac"] < 0.2 or ctas < N_SMS) else "dependent loop of a block and HBM together (see the profile)")
     tr = NCU_TRAFFIC.get(f"config{cfg}", {})
     if tr.get("src_sha") == kernel_src_sha() and not small:
         roof["traffic"] = tr.get("bytes_per_launch")
