@@ -385,18 +385,18 @@ def measure_e2e(ctx, wl, host, n_e2e, world, dev):
     import torch
     import torch.distributed as dist
 
-    Xh, yh = host
     vh = torch.empty(wl.d, dtype=torch.float32, pin_memory=True)
-    args = (Xh, yh, wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    solve = ctx.solve_host_csr if wl.sparse else ctx.solve_host
+    args = tuple(host) + (wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
     for _ in range(2):
-        ctx.solve_host(*args, out=vh)
+        solve(*args, out=vh)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(n_e2e):
-        ctx.solve_host(*args, out=vh)
+        solve(*args, out=vh)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
@@ -405,13 +405,22 @@ def measure_e2e(ctx, wl, host, n_e2e, world, dev):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     return {"value": float(wl.total_steps) * world * n_e2e / (ms * 1e-3), "unit": UNIT,
-            "h2d_bytes_per_step": int(Xh.numel() * Xh.element_size() + yh.numel() * 4) * world,
+            "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host)) * world,
             "d2h_bytes_per_step": int(wl.d * 4) * world, "steps": n_e2e}
 
 
 def pinned_host_rows(wl):
-    """Pinned host copies of a dense workload's rows and labels (chunked, so no second pageable copy is needed)."""
+    """Pinned host copies of a workload's rows and labels (dense rows chunked, so no second pageable copy is needed)."""
     import torch
+
+    if wl.sparse:
+        out = []
+        for t in (wl.row_ptr, wl.col_idx, wl.val, wl.y):
+            h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+            h.copy_(t)
+            out.append(h)
+        torch.cuda.synchronize()
+        return tuple(out)
 
     Xh = torch.empty(wl.X.shape, dtype=wl.X.dtype, pin_memory=True)
     rows = max(1, (1 << 28) // max(1, wl.X.shape[1] * wl.X.element_size()))
@@ -495,9 +504,7 @@ def main():
     # ---- end to end through the host-buffer entry point (dense rows; pinned host memory must hold them) -------------
     e2e = None
     if not args.no_e2e:
-        if wl.sparse:
-            e2e = {"value": None, "unit": UNIT, "note": "the host-buffer entry point takes dense rows only"}
-        elif input_bytes(wl) * 1.2 > host_memory_available():
+        if input_bytes(wl) * 1.2 > host_memory_available():
             e2e = {"value": None, "unit": UNIT,
                    "note": f"host buffer of {input_bytes(wl) / 2**30:.1f} GiB not attempted: "
                            f"{host_memory_available() / 2**30:.1f} GiB of host memory available"}
@@ -541,7 +548,7 @@ def main():
                     ent, ctx2 = measure(P, multi, w2, c2, dev, 10, 3, peak, peak_src, options)
                     if c2 == 5:
                         ent["rho"] = rho
-                    if not w2.sparse and not args.no_e2e and (c2 != 5 or rho == args.rho):
+                    if not args.no_e2e and (c2 != 5 or rho == args.rho):
                         ent["e2e"] = measure_e2e(ctx2, w2, pinned_host_rows(w2), 5, 1, dev)
                     ctx2.destroy()
                     if not args.no_cpu_baseline and (c2 != 5 or rho == args.rho):

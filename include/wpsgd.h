@@ -226,6 +226,14 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* ctx, const void* X, wpsgd_xtype xt, con
                               float lambda, wpsgd_loss loss, uint64_t seed, const float* w0, double r,
                               float* v_out);
 
+/* The same from HOST buffers for CSR rows (the paper's kind of data): row_ptr HOST [N+1], col_idx HOST [nnz], val HOST
+ * [nnz], y HOST [N], w0 HOST [d] or NULL, v_out HOST [d]; other arguments as wpsgd_run_csr and wpsgd_combine. Copies
+ * the arrays to staging buffers of the context, runs the chains and the combination, copies v back and waits. */
+wpsgd_status wpsgd_solve_host_csr(wpsgd_ctx* ctx, const int64_t* row_ptr, const int32_t* col_idx, const float* val,
+                                  const float* y, const int64_t* shard_off, const int64_t* n_steps, float eta0,
+                                  wpsgd_lr sched, float lambda, wpsgd_loss loss, uint64_t seed, const float* w0, double r,
+                                  float* v_out);
+
 /* An entry point for callers that must not allocate device memory. (The paper has no counterpart:
  * this is a convenience of the library.) It does what wpsgd_run followed by wpsgd_combine does on
  * dense rows, but takes no context and calls no cudaMalloc / cudaFree or any other allocating

@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "wpsgd_combine", "wpsgd_combine_weighted", "wpsgd_last_chain_ms", "wpsgd_get_models", "wpsgd_set_models", "wpsgd_get_weights", "wpsgd_weights",
     "wpsgd_sample_indices", "wpsgd_objective", "wpsgd_objective_csr", "wpsgd_solve_host", "wpsgd_solve_static", "wpsgd_check", "wpsgd_launch_count",
     "wpsgd_last_error", "wpsgd_continue_csr", "wpsgd_validate_csr", "wpsgd_span_valid", "wpsgd_sample_indices_host",
-    "wpsgd_check_static",
+    "wpsgd_check_static", "wpsgd_solve_host_csr",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.wpsgd_span_valid.argtypes = [vp, i32, f32, f32, f64, i64, ctypes.POINTER(f64), ctypes.POINTER(ci)]
     lib.wpsgd_sample_indices_host.argtypes = [u64, i32, i64, i64, i64, i32, vp]
     lib.wpsgd_check_static.argtypes = [ci, vp]
+    lib.wpsgd_solve_host_csr.argtypes = [vp, vp, vp, vp, vp, vp, vp, f32, ci, f32, ci, u64, vp, f64, vp]
     lib.wpsgd_launch_count.argtypes = [vp]
     lib.wpsgd_launch_count.restype = i64
     lib.wpsgd_last_error.argtypes = [vp]
@@ -398,6 +399,24 @@ class Context:
                                             ctypes.c_void_p(y.data_ptr()), so.ctypes.data, ns.ctypes.data, eta0, sched,
                                             lam, loss, seed, ctypes.c_void_p(w0.data_ptr()) if w0 is not None else None,
                                             r, ctypes.c_void_p(out.data_ptr())), "wpsgd_solve_host")
+        return out
+
+    def solve_host_csr(self, row_ptr, col_idx, val, y, shard_off, n_steps, eta0, sched, lam, loss, seed, w0=None,
+                       r: float = 0.0, out=None):
+        """Host CSR tensors in (ideally pinned), host tensor out; copies are part of the call."""
+        import torch
+
+        for t, dt in ((row_ptr, torch.int64), (col_idx, torch.int32), (val, torch.float32), (y, torch.float32)):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dt:
+                raise TypeError("solve_host_csr takes contiguous host tensors (int64 row_ptr, int32 col_idx, float32 val, y)")
+        so, ns = _host_i64(shard_off), _host_i64(n_steps)
+        if out is None:
+            out = torch.empty(self.d, dtype=torch.float32).pin_memory()
+        self._ck(self._lib.wpsgd_solve_host_csr(self._h, ctypes.c_void_p(row_ptr.data_ptr()), ctypes.c_void_p(col_idx.data_ptr()),
+                                                ctypes.c_void_p(val.data_ptr()), ctypes.c_void_p(y.data_ptr()),
+                                                so.ctypes.data, ns.ctypes.data, eta0, sched, lam, loss, seed,
+                                                ctypes.c_void_p(w0.data_ptr()) if w0 is not None else None, r,
+                                                ctypes.c_void_p(out.data_ptr())), "wpsgd_solve_host_csr")
         return out
 
     def check(self):

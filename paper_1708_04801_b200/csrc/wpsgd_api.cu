@@ -52,6 +52,12 @@ struct wpsgd_ctx {
   float* st_y = nullptr;
   size_t st_y_cap = 0;
   float* st_v = nullptr;   // [d]
+  long long* st_rp = nullptr;  // CSR staging of the host-buffer entry point
+  size_t st_rp_cap = 0;
+  int* st_ci = nullptr;
+  size_t st_ci_cap = 0;
+  float* st_va = nullptr;
+  size_t st_va_cap = 0;
   float* st_w0 = nullptr;  // [d]
   // state of the chains
   bool have_run = false;
@@ -838,7 +844,7 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* c) {
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
   void* ptrs[] = {c->W, c->scale, c->t_shard_off, c->t_steps, c->t_first, c->t_idx_off, c->t_rows, c->t_count, c->t_order,
-                  c->t_ids, c->t_group, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0};
+                  c->t_ids, c->t_group, c->t_weights, c->idx, c->status, c->part, c->st_X, c->st_y, c->st_v, c->st_w0, c->st_rp, c->st_ci, c->st_va};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev0) cudaEventDestroy(c->ev0);
@@ -1201,6 +1207,46 @@ wpsgd_status wpsgd_solve_host(wpsgd_ctx* c, const void* X, wpsgd_xtype xt, const
                          w0 ? c->st_w0 : nullptr, false, &groups);
     if (s != WPSGD_OK) return s;
   }
+  s = wpsgd_combine(c, r, c->st_v);
+  if (s != WPSGD_OK) return s;
+  CU_TRY(c, cudaMemcpyAsync(v_out, c->st_v, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CU_TRY(c, cudaStreamSynchronize(c->stream));
+  return WPSGD_OK;
+}
+
+wpsgd_status wpsgd_solve_host_csr(wpsgd_ctx* c, const int64_t* row_ptr, const int32_t* col_idx, const float* val, const float* y,
+                                  const int64_t* shard_off, const int64_t* n_steps, float eta0, wpsgd_lr sched, float lambda,
+                                  wpsgd_loss loss, uint64_t seed, const float* w0, double r, float* v_out) {
+  if (!c) return fail(nullptr, WPSGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!shard_off || !v_out) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off or v_out is NULL");
+  DeviceGuard guard(c->device);
+  const long long N = shard_off[c->k];
+  if (N < 0) return fail(c, WPSGD_ERR_INVALID_ARG, "shard_off[k] < 0");
+  if (N > 0 && (!row_ptr || !y)) return fail(c, WPSGD_ERR_INVALID_ARG, "row_ptr or y is NULL");
+  const long long nnz = N > 0 ? row_ptr[N] : 0;
+  if (nnz < 0 || (nnz > 0 && (!col_idx || !val))) return fail(c, WPSGD_ERR_INVALID_ARG, "row_ptr[N] < 0, or col_idx / val is NULL");
+  wpsgd_status s = grow(c, &c->st_rp, &c->st_rp_cap, (size_t)N + 1);
+  if (s != WPSGD_OK) return s;
+  s = grow(c, &c->st_ci, &c->st_ci_cap, (size_t)std::max(1ll, nnz));
+  if (s != WPSGD_OK) return s;
+  s = grow(c, &c->st_va, &c->st_va_cap, (size_t)std::max(1ll, nnz));
+  if (s != WPSGD_OK) return s;
+  s = grow(c, &c->st_y, &c->st_y_cap, (size_t)std::max(1ll, N));
+  if (s != WPSGD_OK) return s;
+  if (!c->st_v) CU_TRY(c, cudaMalloc((void**)&c->st_v, (size_t)c->d * sizeof(float)));
+  if (w0 && !c->st_w0) CU_TRY(c, cudaMalloc((void**)&c->st_w0, (size_t)c->d * sizeof(float)));
+  if (N > 0) {
+    CU_TRY(c, cudaMemcpyAsync(c->st_rp, row_ptr, ((size_t)N + 1) * sizeof(long long), cudaMemcpyHostToDevice, c->stream));
+    CU_TRY(c, cudaMemcpyAsync(c->st_y, y, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  }
+  if (nnz > 0) {
+    CU_TRY(c, cudaMemcpyAsync(c->st_ci, col_idx, (size_t)nnz * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    CU_TRY(c, cudaMemcpyAsync(c->st_va, val, (size_t)nnz * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  }
+  if (w0) CU_TRY(c, cudaMemcpyAsync(c->st_w0, w0, (size_t)c->d * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  s = wpsgd_run_csr(c, (const int64_t*)c->st_rp, c->st_ci, c->st_va, c->st_y, shard_off, n_steps, eta0, sched, lambda, loss, seed,
+                    w0 ? c->st_w0 : nullptr);
+  if (s != WPSGD_OK) return s;
   s = wpsgd_combine(c, r, c->st_v);
   if (s != WPSGD_OK) return s;
   CU_TRY(c, cudaMemcpyAsync(v_out, c->st_v, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));

@@ -589,6 +589,20 @@ def test_solve_host_pipelined_equals_device_path(P, d, bf16, k, pipeline):
         ctx.check()
 
 
+def test_solve_host_csr_equals_device_path(P):
+    wl = wi.config4(k=5, d=4096, m=200, base_steps=500, mean_nnz=25.0)
+    wl.w0 = torch.full((4096,), 0.02)
+    v_dev, _, _, _ = gpu_solve(P, wl)
+    with P.Context(wl.k, wl.d) as ctx:
+        for _ in range(2):
+            out = ctx.solve_host_csr(wl.row_ptr.pin_memory(), wl.col_idx.pin_memory(), wl.val.pin_memory(), wl.y.pin_memory(),
+                                     wl.shard_off, wl.n_steps, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed, w0=wl.w0)
+            np.testing.assert_array_equal(out.numpy(), v_dev)
+        ctx.check()
+    ov, _, _ = oracle.solve(wl)
+    assert rel_l2(out.numpy(), ov) <= TOL[wl.loss]
+
+
 # ---- sparse path --------------------------------------------------------------------------------------------
 # sparse_variant 1: one step per round trip to the model in global memory; 2 (the default): blocks of steps run in a
 # shared-memory cache of the model entries they touch
