@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <functional>
 #include <numeric>
 #include <string>
 #include <vector>
@@ -479,6 +480,34 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   }
 }
 
+// Warp-per-node kernel: one CTA of four warps per SM, or two? A warp alone on its scheduler takes about 2640 cycles
+// per block of 8 samples, two warps sharing one about 3000 each (measured, k = 1024, d = 256). With one CTA per SM
+// there are 148 CTA slots and the remaining CTAs queue behind, longest first; with two there are 296 slots. Which
+// finishes first depends on the step counts (equal work: 3.57 ms with two against 5.28 ms with one; speed ratio 16:
+// 5.69 ms against 4.97 ms), so both schedules are played through on the host: CTAs in launch order (a CTA lasts as long
+// as its longest chain) onto the slot that frees first.
+bool two_warp_ctas_per_sm_finish_first(const std::vector<long long>& steps, int warps) {
+  std::vector<long long> sorted(steps);
+  std::sort(sorted.begin(), sorted.end(), [](long long a, long long b) { return a > b; });
+  std::vector<long long> cta_cost;
+  for (size_t i = 0; i < sorted.size(); i += (size_t)warps) cta_cost.push_back(sorted[i]);
+  auto makespan = [&](int slots, double cycles_per_block) {
+    std::vector<double> free_at((size_t)std::min<size_t>((size_t)slots, cta_cost.size()), 0.0);
+    if (free_at.empty()) return 0.0;
+    std::make_heap(free_at.begin(), free_at.end(), std::greater<double>());
+    double end = 0.0;
+    for (long long cost : cta_cost) {
+      std::pop_heap(free_at.begin(), free_at.end(), std::greater<double>());
+      const double t = free_at.back() + (double)cost * cycles_per_block;
+      free_at.back() = t;
+      end = std::max(end, t);
+      std::push_heap(free_at.begin(), free_at.end(), std::greater<double>());
+    }
+    return end;
+  };
+  return makespan(2 * 148, 3000.0) < makespan(148, 2640.0);
+}
+
 // blocked kernel, one warp per node (small d)
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, int nk, bool aligned, int* R_out, int* stages_out, int* warps_out) {
@@ -496,10 +525,8 @@ bool block_warp_kernel_fits(const wpsgd_ctx* c, int nk, bool aligned, int* R_out
   if (nk != c->k) return false;  // its node-to-CTA table covers the whole node set
   int warps = (int)std::min<long long>(4, std::max<long long>(1, nk));
   if (c->opt_threads >= 32 && c->opt_threads % 32 == 0) warps = std::min(BLKW_MAX_WARPS, c->opt_threads / 32);
-  // With at least four chains per SM in all, one CTA per SM (a ring of 4 stages per warp takes the shared memory of a
-  // second one) and the remaining CTAs queued behind, longest first, does a little better than two CTAs per SM
-  // (k = 1024: 4.76 ms against 4.98 ms): a warp alone on its scheduler takes about 2640 cycles per block, 3000 shared.
-  const bool one_cta_per_sm = c->opt_stages >= 4 || (c->opt_stages == 0 && nk >= 4 * 148);
+  // one CTA per SM (a ring of 4 stages per warp takes the shared memory of a second one) or two (3 stages): see above
+  const bool one_cta_per_sm = c->opt_stages >= 4 || (c->opt_stages == 0 && !two_warp_ctas_per_sm_finish_first(c->last_steps, warps));
   int stages = c->opt_stages > 0 ? std::min(c->opt_stages, 4) : (one_cta_per_sm ? 4 : 3);
   while (BlockWarpSmem(stages, row_bytes, warps).total > ((warps <= 4 && !one_cta_per_sm) ? 100 * 1024 : kSmemBudget)) {
     if (stages > 2) --stages;
