@@ -1,4 +1,4 @@
-// Per-node SGD chains on dense rows, blocked form (constant step size).
+// Per-node SGD chains on dense rows, blocked form (constant step size, or eta0 / sqrt(n) with per-block tables).
 //
 // Eq. 5 is a strictly serial recurrence, w_n = a w_{n-1} - eta g_n x_n with a = 1 - eta lambda and
 // g_n = L'(y_n, w_{n-1}.x_n). Taking B consecutive samples x_0..x_{B-1} of a chain together and unrolling,
@@ -225,6 +225,37 @@ constexpr int BLK_B = 8;                           // samples per block
 constexpr int BLK_PAIRS = BLK_B * (BLK_B - 1) / 2;  // 28 Gram entries below the diagonal
 constexpr int BLK_MAX_MATH_WARPS = 16;
 
+// Tables of a block for the decaying schedule eta_n = eta0 / sqrt(n). With a_s = 1 - eta_s lambda and A_m the product
+// of a_s over the block's first m steps: apw[m] = A_m, cfac[m] = eta_m / A_{m+1}, a_nv = A_nv, dl_nv = 1 - A_nv, and
+// apw_own = A of the sample this lane looks after (lane mod B). n0 = steps the chain has run before the block. Formed
+// in fp64 by the lanes of the calling warp and rounded once; all lanes of the warp must call it. (For a constant step
+// size these are powers of a = 1 - eta lambda, kept in shared memory.) The blocked algebra itself does not change:
+// w after n samples = A_n (w_0 - sum_{m<n} beta_m x_m) with beta_m = eta_m g_m / A_{m+1}.
+template <int B>
+__device__ __forceinline__ void decaying_block_tables(double eta0, double lam, long long n0, int nv, float (&apw)[B],
+                                                      float (&cfac)[B], float& apw_own, float& a_nv, float& dl_nv) {
+  const int m = (int)(threadIdx.x & (B - 1));
+  const double eta = eta0 / sqrt((double)(n0 + m + 1));
+  double ia = 1.0 - eta * lam;  // becomes A_{m+1}: inclusive product over the block's steps 0..m
+#pragma unroll
+  for (int o = 1; o < B; o <<= 1) {
+    const double v = __shfl_up_sync(0xffffffffu, ia, o, B);
+    if (m >= o) ia *= v;
+  }
+  double ea = __shfl_up_sync(0xffffffffu, ia, 1, B);  // A_m
+  if (m == 0) ea = 1.0;
+  const double cf = eta / ia;
+#pragma unroll
+  for (int q = 0; q < B; ++q) {
+    apw[q] = (float)__shfl_sync(0xffffffffu, ea, q, B);
+    cfac[q] = (float)__shfl_sync(0xffffffffu, cf, q, B);
+  }
+  const double a_end = nv > 0 ? __shfl_sync(0xffffffffu, ia, nv - 1, B) : 1.0;
+  apw_own = (float)ea;
+  a_nv = (float)a_end;
+  dl_nv = (float)(1.0 - a_end);
+}
+
 // Per-sample constants of a block of 8 with everything folded in that does not depend on the chain:
 // t_n = sc_n (p_n - sum_m beta_m G_mn) is the argument of the loss derivative, beta_n = cf_n * f(t_n).
 // apw[m] = a^m, cfac[m] = eta / a^{m+1}; samples from nv on lie beyond the chain's end and take no step.
@@ -389,13 +420,16 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
     float apw[B], cfac[B];
 #pragma unroll
     for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+    const bool decaying = p.sched == LR_INV_SQRT;
+    const long long first_j = p.first ? p.first[j] : 0;
 
     for (long long b = 0; b < nb; ++b) {
       const int nv = (int)((n_run - b * B) < (long long)B ? (n_run - b * B) : (long long)B);
       const float y_cur = y_nxt;
       if (b + 1 < nb) y_nxt = yshard[id_nxt];
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
-      const float a_nv = tab[nv], dl_nv = tab[32 + nv];
+      float a_nv = tab[nv], dl_nv = tab[32 + nv], apw_own = tab[n];
+      if (decaying) decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl_nv);
       float yv[B], sc[B], cf[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
@@ -442,7 +476,7 @@ __global__ void __launch_bounds__(64 + 32 * MAXW, 1) chain_block_kernel(const Bl
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
-      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * psum, jets, beta);
+      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * apw_own * 1.4426950408889634f * psum, jets, beta);
       // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}
       float mine = dl_nv;
 #pragma unroll
@@ -750,6 +784,8 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
   float apw[B], cfac[B];
 #pragma unroll
   for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+  const bool decaying = p.sched == LR_INV_SQRT;
+  const long long first_j = p.first ? p.first[j] : 0;
 
   bool act[R];
   float w[R][V];
@@ -873,7 +909,8 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
     const float pv_own = scratch[32 + n];  // margin of the sample this lane looks after
     __syncwarp();
     // ---- 8-step recurrence, every lane the same ----------------------------------------------------------
-    const float a_nv = tab[nv], dl = tab[32 + nv];
+    float a_nv = tab[nv], dl = tab[32 + nv], apw_own = tab[n];
+    if (decaying) decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl);
     float t[B], beta[B], yv[B], cf[B], sc[B];
 #pragma unroll
     for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
@@ -885,7 +922,7 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
       for (int k2 = 0; k2 < m; ++k2) Gs[m * (m - 1) / 2 + k2] *= sc[m];
     }
     // lane n & 7 expands the logistic factor of its own sample around t0_n (scratch[40..71] holds the expansions)
-    block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * pv_own, (float4*)(scratch + 40), beta);
+    block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * apw_own * 1.4426950408889634f * pv_own, (float4*)(scratch + 40), beta);
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m,  gamma_m = beta_m a^nv ----------------------------------
     {
       constexpr int NP = XPairs<XT>::NP;

@@ -199,6 +199,8 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
     float apw[B], cfac[B];
 #pragma unroll
     for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
+    const bool decaying = p.sched == LR_INV_SQRT;
+    const long long first_j = p.first ? p.first[j] : 0;
     const uint32_t expect_bytes = C * (uint32_t)math_warps * MMA_SLOT_BYTES;
     cluster_barrier();  // start-up: every CTA of the cluster runs and has set up its shared memory
 
@@ -209,7 +211,8 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
       const float y_cur = y_nxt;
       if (b + 1 < nb) y_nxt = yshard[id_nxt];
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
-      const float a_nv = tab[nv], dl_nv = tab[32 + nv];
+      float a_nv = tab[nv], dl_nv = tab[32 + nv], apw_own = tab[n];
+      if (decaying) decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl_nv);
       float yv[B], sc[B], cf[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
@@ -261,7 +264,7 @@ __global__ void __launch_bounds__(NPL == 4 ? 64 + 32 * 8 : 64 + 32 * 16, 1) chai
       float t[B], beta[B];
 #pragma unroll
       for (int m = 0; m < B; ++m) t[m] = sc[m] * __shfl_sync(0xffffffffu, psum, m);
-      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * tab[n] * 1.4426950408889634f * psum, jets, beta);
+      block8_recurrence<LOSS>(t, Gs, cf, yv, y_cur * apw_own * 1.4426950408889634f * psum, jets, beta);
       // gamma_m = eta g_m a^{nv-1-m} = beta_m a^{nv}; [8] = 1 - a^nv; [9] = leave after this block
       float mine = dl_nv;
 #pragma unroll

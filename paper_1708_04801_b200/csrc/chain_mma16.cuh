@@ -124,6 +124,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
     if (nb > 0) y_nxt = yshard[idx[n]];
     if (nb > 1) id_nxt = idx[B + n];
     const uint32_t expect_bytes = C * (uint32_t)math_warps * M16_SLOT_BYTES;
+    const bool decaying = p.sched == LR_INV_SQRT;
+    const long long first_j = p.first ? p.first[j] : 0;
     cluster_barrier();  // start-up: every CTA of the cluster runs and has set up its shared memory
 
     for (long long b = 0; b < nb; ++b) {
@@ -133,7 +135,15 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       const float y_cur = y_nxt;  // lane l: label of sample l & 15
       if (b + 1 < nb) y_nxt = yshard[id_nxt];
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
-      const float a_nv = tab[nv], dl_nv = tab[64 + nv];
+      float a_nv = tab[nv], dl_nv = tab[64 + nv];
+      float apw[B], cfac[B];
+      if (decaying) {
+        float apw_own;
+        decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl_nv);
+      } else {
+#pragma unroll
+        for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[32 + m]; }
+      }
       // ---- wait (bounded) for the partial sums of block b from every math warp of the cluster ------------------
       {
         const uint32_t parity = (uint32_t)((b >> 1) & 1);
@@ -171,13 +181,12 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
 #pragma unroll
       for (int m = 0; m < B; ++m) {
         yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
-        const float apw = tab[m], cfac = tab[32 + m];
         if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
-          sc[m] = yv[m] * apw;
-          cf[m] = -yv[m] * cfac;
+          sc[m] = yv[m] * apw[m];
+          cf[m] = -yv[m] * cfac[m];
         } else {  // squared: g = t - y, t = a^n (...)
-          sc[m] = apw;
-          cf[m] = cfac;
+          sc[m] = apw[m];
+          cf[m] = cfac[m];
         }
         if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
       }

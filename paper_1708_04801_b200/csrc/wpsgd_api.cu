@@ -326,7 +326,7 @@ constexpr size_t kSmemBudget = 220 * 1024;
 template <typename XT>
 bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* R_out, int* stages_out) {
   constexpr int V = XVec<XT>::V;
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if (!aligned) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;  // keeps a^-8 harmless in fp32
   const long long chunks = c->d / V;
   // up to 8 math warps with one chunk per thread (two register copies of a block: Gram products overlap the
@@ -398,7 +398,7 @@ struct ClusterShape {
 };
 
 bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if (!aligned) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
   const long long chunks = c->d / 8;
   if (chunks < 1) return false;
@@ -512,7 +512,7 @@ bool two_warp_ctas_per_sm_finish_first(const std::vector<long long>& steps, int 
 template <typename XT>
 bool block_warp_kernel_fits(const wpsgd_ctx* c, int nk, bool aligned, int* R_out, int* stages_out, int* warps_out) {
   constexpr int V = XVec<XT>::V;
-  if (!aligned || c->sched != WPSGD_LR_CONST) return false;
+  if (!aligned) return false;
   if ((double)c->eta0 * (double)c->lambda > 0.25) return false;
   const long long chunks = c->d / V;
   const int R = (int)((chunks + 31) / 32);
@@ -607,7 +607,7 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   if (variant == 5) {
     if (!block_warp_ok)
       return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, a constant step size and "
+                  "blocked warp kernel needs 16-byte aligned rows of at most 64 chunks, "
                   "eta*lambda <= 0.25");
     return launch_block_warp<XT>(c, p, wR, wstages, wwarps);
   }
@@ -615,14 +615,14 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
     ClusterShape sh;
     if (sizeof(XT) != 2 || !mma_kernel_fits(c, aligned, &sh))
       return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "tensor-core cluster kernel needs bf16 rows, 16-byte aligned, a constant step size, eta*lambda <= 0.25, a "
+                  "tensor-core cluster kernel needs bf16 rows, 16-byte aligned, eta*lambda <= 0.25, a "
                   "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
     return launch_mma(c, p, sh);
   }
   if (variant == 4) {
     if (!block_ok)
       return fail(c, WPSGD_ERR_UNSUPPORTED,
-                  "blocked kernel needs 16-byte aligned rows of at most 8 KiB, a constant step size and eta*lambda <= 0.25");
+                  "blocked kernel needs 16-byte aligned rows of at most 8 KiB and eta*lambda <= 0.25");
     return launch_block<XT>(c, p, bthreads, bR, bstages);
   }
   if ((variant == 2 || variant == 3) && !aligned)

@@ -114,15 +114,10 @@ def test_dense_variants(P, variant, threads, prefetch, bf16):
 
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
 @pytest.mark.parametrize("sched", [0, 1])
-@pytest.mark.parametrize("variant", [1, 2, 3, 4])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5])
 def test_losses_and_schedules(P, loss, sched, variant):
     wl = wi.config1(k=3, d=64, m=128, n_steps=(300, 150, 40))
     wl.loss, wl.sched = loss, sched
-    if variant == 4 and sched == 1:  # the blocked kernel is for the constant step size
-        with pytest.raises(P.WpsgdError) as e:
-            gpu_solve(P, wl, {"dense_variant": 4})
-        assert e.value.status_name == "UNSUPPORTED"
-        return
     wl.eta0 = 0.05 if sched else 0.01
     if loss == SQUARED:
         wl.y = (wl.y * 0.5 + 0.1).contiguous()
@@ -155,6 +150,43 @@ def test_generic_kernel_handles_unaligned_shapes(P):
 def test_large_d_falls_back_and_matches(P):
     wl = wi.config2(k=2, d=8200, m=16, base_steps=40)  # beyond the register kernels' reach
     assert_parity(P, wl)
+
+
+# ---- blocked kernels with the decaying step size eta0 / sqrt(n): per-block tables instead of powers of one factor -------
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+@pytest.mark.parametrize("kind", ["block_fp32", "block_bf16", "warp", "mma8", "mma16"])
+def test_blocked_kernels_decaying_step_size(P, kind, loss):
+    if kind == "mma16" and loss == LOGISTIC:
+        pytest.skip("the 16-sample form has squared and hinge losses only")
+    d = {"block_fp32": 1024, "block_bf16": 1000, "warp": 256, "mma8": 2048, "mma16": 2048}[kind]
+    wl = wi.config2(k=4, d=d, m=96, base_steps=333)
+    wl.n_steps[3] = 0
+    wl.loss, wl.sched, wl.eta0, wl.lam = loss, 1, 0.3, 0.05  # eta_n lambda from 1.5e-2 down: the factors differ step by step
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    wl.w0 = torch.full((d,), 0.05)
+    if kind != "block_fp32" and kind != "warp":
+        wl.X = wl.X.to(torch.bfloat16)
+    opts = {"block_fp32": {"dense_variant": 4}, "block_bf16": {"dense_variant": 4}, "warp": {"dense_variant": 5},
+            "mma8": {"dense_variant": 8, "block_samples": 8, "cluster": 2},
+            "mma16": {"dense_variant": 8, "block_samples": 16, "cluster": 2}}[kind]
+    assert_parity(P, wl, opts)
+
+
+def test_decaying_step_size_continue_keeps_the_step_numbers(P):
+    # a continued chain must take eta of its own step numbers (first + n), also inside the per-block tables
+    wl_cpu = wi.config2(k=3, d=1024, m=64, base_steps=8)
+    wl_cpu.n_steps = np.array([203, 101, 50], dtype=np.int64)
+    wl_cpu.sched, wl_cpu.eta0, wl_cpu.lam = 1, 0.3, 0.05
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.run(wl.X, wl.y, wl.shard_off, np.array([50, 50, 50]), wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        ctx.continue_(wl.X, wl.y, wl.shard_off, np.array([153, 51, 0]))
+        seg = ctx.get_models().cpu().numpy()
+        ctx.check()
+    oW = oracle.run_dense(wl_cpu.X, wl_cpu.y, wl.shard_off, wl_cpu.n_steps, wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    for j in range(wl.k):
+        assert rel_l2(seg[j], oW[j]) <= 1e-4
 
 
 # ---- blocked kernel: block boundaries, ring depths, column tilings ----------------------------------------
