@@ -235,8 +235,13 @@ template <int B>
 __device__ __forceinline__ void decaying_block_tables(double eta0, double lam, long long n0, int nv, float (&apw)[B],
                                                       float (&cfac)[B], float& apw_own, float& a_nv, float& dl_nv) {
   const int m = (int)(threadIdx.x & (B - 1));
-  const double eta = eta0 / sqrt((double)(n0 + m + 1));
-  double ia = 1.0 - eta * lam;  // becomes A_{m+1}: inclusive product over the block's steps 0..m
+  // 1 / sqrt(n) and 1 / A from the fp32 special-function unit plus one Newton step in fp64 (relative error below
+  // 1e-12): no fp64 square root or division on the way
+  const double nn = (double)(n0 + m + 1);
+  double rs = (double)rsqrtf((float)nn);
+  rs = rs * fma(-0.5 * nn, rs * rs, 1.5);
+  const double eta = eta0 * rs;
+  double ia = fma(-eta, lam, 1.0);  // becomes A_{m+1}: inclusive product over the block's steps 0..m
 #pragma unroll
   for (int o = 1; o < B; o <<= 1) {
     const double v = __shfl_up_sync(0xffffffffu, ia, o, B);
@@ -244,14 +249,16 @@ __device__ __forceinline__ void decaying_block_tables(double eta0, double lam, l
   }
   double ea = __shfl_up_sync(0xffffffffu, ia, 1, B);  // A_m
   if (m == 0) ea = 1.0;
-  const double cf = eta / ia;
+  double rc = (double)__frcp_rn((float)ia);
+  rc = rc * fma(-ia, rc, 2.0);
+  const float apw_f = (float)ea, cf_f = (float)(eta * rc);
 #pragma unroll
   for (int q = 0; q < B; ++q) {
-    apw[q] = (float)__shfl_sync(0xffffffffu, ea, q, B);
-    cfac[q] = (float)__shfl_sync(0xffffffffu, cf, q, B);
+    apw[q] = __shfl_sync(0xffffffffu, apw_f, q, B);
+    cfac[q] = __shfl_sync(0xffffffffu, cf_f, q, B);
   }
   const double a_end = nv > 0 ? __shfl_sync(0xffffffffu, ia, nv - 1, B) : 1.0;
-  apw_own = (float)ea;
+  apw_own = apw_f;
   a_nv = (float)a_end;
   dl_nv = (float)(1.0 - a_end);
 }
