@@ -31,16 +31,18 @@ constexpr int M16_B = 16;
 constexpr int M16_PAIRS = M16_B * (M16_B - 1) / 2;  // 120
 constexpr int M16_SLOT_FLOATS = 256;   // D0 [16][8] | D1 rows 8..15 [8][8] | p parts [16][4]
 constexpr uint32_t M16_SLOT_BYTES = M16_SLOT_FLOATS * sizeof(float);
-constexpr int M16_SLOTS = 16;          // math warps of a whole cluster
+constexpr int M16_SLOTS = 8;           // one slot per CTA of the cluster
+constexpr int M16_WARPS = 8;           // math warps of a CTA
 
 struct Mma16Smem {
-  size_t row_stride, ring, w3, red, tot, gam, tab, bars, pbar, flag, total;
+  size_t row_stride, ring, w3, red, part, tot, gam, tab, bars, pbar, flag, total;
   __host__ __device__ Mma16Smem(int stages, size_t slice_bytes) {
     row_stride = slice_bytes + 16;
     ring = 0;
     w3 = ring + (size_t)stages * M16_B * row_stride;                 // w_hi, w_mid, w_lo, one zero row
     red = w3 + 4 * row_stride;                                       // [2][slots][256] partial sums
-    tot = red + 2 * (size_t)M16_SLOTS * M16_SLOT_FLOATS * sizeof(float);  // [256] sums over the slots
+    part = red + 2 * (size_t)M16_SLOTS * M16_SLOT_FLOATS * sizeof(float);  // [math warps][256] this CTA's partial sums
+    tot = part + (size_t)M16_WARPS * M16_SLOT_FLOATS * sizeof(float);      // [256] sums over the slots
     gam = tot + M16_SLOT_FLOATS * sizeof(float);                     // gamma_0..15, 1 - a^nv, stop
     tab = gam + 32 * sizeof(float);                                  // [3][32]
     bars = tab + 3 * 32 * sizeof(float);                             // ring barriers [8]
@@ -49,6 +51,13 @@ struct Mma16Smem {
     total = flag + 16;
   }
 };
+
+// 16-byte store into the shared memory of a CTA of the cluster, counted on that CTA's barrier `mbar`
+__device__ __forceinline__ void st_async_f32x4(uint32_t addr, float4 v, uint32_t mbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+               "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(mbar)
+               : "memory");
+}
 
 __device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], const void* smem_ptr) {
   const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_ptr);
@@ -79,6 +88,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   unsigned char* ring = smem + L.ring;
   unsigned char* w3 = smem + L.w3;
   float* red = (float*)(smem + L.red);
+  float* part = (float*)(smem + L.part);
   float* tot = (float*)(smem + L.tot);
   float* gam = (float*)(smem + L.gam);   // [0..15] gamma, [16] = 1 - a^nv, [17] = leave after this block
   float* tab = (float*)(smem + L.tab);   // [0..16] a^k, [32..48] eta / a^{k+1}, [64..80] 1 - a^k
@@ -123,7 +133,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
     uint32_t id_nxt = 0u;
     if (nb > 0) y_nxt = yshard[idx[n]];
     if (nb > 1) id_nxt = idx[B + n];
-    const uint32_t expect_bytes = C * (uint32_t)math_warps * M16_SLOT_BYTES;
+    const uint32_t expect_bytes = C * M16_SLOT_BYTES;
     const bool decaying = p.sched == LR_INV_SQRT;
     const long long first_j = p.first ? p.first[j] : 0;
     cluster_barrier();  // start-up: every CTA of the cluster runs and has set up its shared memory
@@ -164,6 +174,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
         float4 s0 = r4[lane], s1 = r4[32 + lane];
 #pragma unroll
         for (int w = 1; w < M16_SLOTS; ++w) {
+          if ((uint32_t)w >= C) break;
           const float4 v0 = r4[w * (M16_SLOT_FLOATS / 4) + lane], v1 = r4[w * (M16_SLOT_FLOATS / 4) + 32 + lane];
           s0.x += v0.x; s0.y += v0.y; s0.z += v0.z; s0.w += v0.w;
           s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
@@ -344,7 +355,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   const size_t warp_col_bytes = (size_t)mw * 512;
   const size_t x_off = (size_t)((lane & 7) + 8 * ((lane >> 3) & 1)) * row_stride + warp_col_bytes + (size_t)(lane >> 4) * 16;
   const unsigned char* w_src = w3 + (size_t)((lane & 7) < 3 ? (lane & 7) : 3) * row_stride + warp_col_bytes + (size_t)((lane >> 3) & 1) * 16;
-  const int slot = (int)rank * math_warps + mw;
   // shared-memory window of every CTA of the cluster (the same offsets apply inside each window)
   const uint32_t own_base = (uint32_t)__cvta_generic_to_shared(smem);
   uint32_t peer_base[8];
@@ -361,7 +371,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
     }
   };
   // D0, D1, D2 of a block over this warp's columns, sent to this warp's slot of every CTA of the cluster
-  auto tensor_pass = [&](const unsigned char* stage, int q) __attribute__((always_inline)) {
+  auto tensor_pass = [&](const unsigned char* stage, int q, uint4 (&raw)[B]) __attribute__((always_inline)) {
     float d0[2][4], d1[2][4], d2[2][4];  // two independent accumulator sets (a dependent mma takes about 20 cycles)
 #pragma unroll
     for (int a = 0; a < 2; ++a)
@@ -377,6 +387,13 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
           ldmatrix_x4(xa[a], xs + (size_t)(round * 2 + a) * 32);
           ldmatrix_x2(wb[a], w_src + (size_t)(round * 2 + a) * 32);
         }
+      // this thread's columns of two of the 16 rows, for the update: between the tensor-core steps these loads find the
+      // shared-memory pipe idle; after the pass they would queue ahead of the sums that the recurrence warp waits for
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        const int m = round * 2 + a;
+        raw[m] = act ? *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16) : make_uint4(0u, 0u, 0u, 0u);
+      }
 #pragma unroll
       for (int a = 0; a < 2; ++a)
         if (round * 2 + a < ksteps) {
@@ -391,26 +408,33 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       d1[0][e] += d1[1][e];
       d2[0][e] += d2[1][e];
     }
-    // accumulator (row g8 / g8 + 8, columns 2 t4, 2 t4 + 1)
-    float* sl = red + ((size_t)q * M16_SLOTS + slot) * M16_SLOT_FLOATS;
-    const uint32_t o0a = (uint32_t)__cvta_generic_to_shared(sl + g8 * 8 + 2 * t4) - own_base;
-    const uint32_t o0b = (uint32_t)__cvta_generic_to_shared(sl + (g8 + 8) * 8 + 2 * t4) - own_base;
-    const uint32_t o1 = (uint32_t)__cvta_generic_to_shared(sl + 128 + g8 * 8 + 2 * t4) - own_base;
-    const uint32_t o2a = (uint32_t)__cvta_generic_to_shared(sl + 192 + g8 * 4 + 2 * t4) - own_base;
-    const uint32_t o2b = (uint32_t)__cvta_generic_to_shared(sl + 192 + (g8 + 8) * 4 + 2 * t4) - own_base;
+    asm volatile("bar.arrive 2, %0;" ::"r"(consumed_threads) : "memory");  // this warp is done with the stage of the block
+    // Two-level sum. Each warp puts its accumulators (row g8 / g8 + 8, columns 2 t4, 2 t4 + 1) into its own table of
+    // this CTA; after a barrier among the math warps the first 64 math threads add the tables up in a fixed order,
+    // 16 bytes each, and send the CTA's sums to this CTA's slot in every CTA of the cluster.
+    float* sl = part + (size_t)mw * M16_SLOT_FLOATS;
+    *(float2*)(sl + g8 * 8 + 2 * t4) = make_float2(d0[0][0], d0[0][1]);
+    *(float2*)(sl + (g8 + 8) * 8 + 2 * t4) = make_float2(d0[0][2], d0[0][3]);
+    *(float2*)(sl + 128 + g8 * 8 + 2 * t4) = make_float2(d1[0][2], d1[0][3]);
+    if (t4 < 2) {  // columns 0..3 of D2: the three parts of p and the zero row
+      *(float2*)(sl + 192 + g8 * 4 + 2 * t4) = make_float2(d2[0][0], d2[0][1]);
+      *(float2*)(sl + 192 + (g8 + 8) * 4 + 2 * t4) = make_float2(d2[0][2], d2[0][3]);
+    }
+    asm volatile("bar.sync 3, %0;" ::"r"(math_warps * 32) : "memory");
     const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&pbar[q]) - own_base;
+    for (int e = mw * 32 + lane; e < M16_SLOT_FLOATS / 4; e += math_warps * 32) {
+      const float4* p4 = (const float4*)part + e;
+      float4 sum = p4[0];
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) {
-      if ((uint32_t)rr < C) {
-        const uint32_t pb = peer_base[rr];
-        st_async_f32x2(pb + o0a, d0[0][0], d0[0][1], pb + ob);
-        st_async_f32x2(pb + o0b, d0[0][2], d0[0][3], pb + ob);
-        st_async_f32x2(pb + o1, d1[0][2], d1[0][3], pb + ob);
-        if (t4 < 2) {  // columns 0..3 of D2: the three parts of p and the zero row
-          st_async_f32x2(pb + o2a, d2[0][0], d2[0][1], pb + ob);
-          st_async_f32x2(pb + o2b, d2[0][2], d2[0][3], pb + ob);
+      for (int w = 1; w < M16_WARPS; ++w)
+        if (w < math_warps) {
+          const float4 v = p4[w * (M16_SLOT_FLOATS / 4)];
+          sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
-      }
+      const uint32_t od = (uint32_t)__cvta_generic_to_shared(red + ((size_t)q * M16_SLOTS + rank) * M16_SLOT_FLOATS + 4 * e) - own_base;
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr)
+        if ((uint32_t)rr < C) st_async_f32x4(peer_base[rr] + od, sum, peer_base[rr] + ob);
     }
   };
 
@@ -419,12 +443,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   for (long long b = 0; b < nb; ++b) {
     wait_rows(st, par);
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
-    tensor_pass(stage, (int)(b & 1));
-    // this thread's columns of the 16 rows, for the update: afterwards the stage can be refilled
-    uint4 raw[B];
-#pragma unroll
-    for (int m = 0; m < B; ++m) raw[m] = act ? *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16) : make_uint4(0u, 0u, 0u, 0u);
-    asm volatile("bar.arrive 2, %0;" ::"r"(consumed_threads) : "memory");  // this warp is done with the stage of block b
+    uint4 raw[B];  // this thread's columns of the 16 rows, for the update
+    tensor_pass(stage, (int)(b & 1), raw);
     __syncthreads();  // gamma_b and the decision are in gam; every math warp is done with the stage of block b
     if (gam[B + 1] != 0.0f) break;
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m, then the model rows again -----------------------------------------
