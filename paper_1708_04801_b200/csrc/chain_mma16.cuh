@@ -14,13 +14,19 @@
 //     D2 = X [w_hi w_mid w_lo 0 ..]^T (16 x 8)   columns 0..2: the three parts of p_n = w . x_n
 // with exact bf16 products and fp32 accumulation. 48 bytes of operand reads per sample and 16 columns instead of 64.
 //
-// One block ahead. The Gram part (D0, D1) does not depend on the model, so the math warps form it for block b + 1
-// while the recurrence warp works on block b; the A-tile registers stay for the margin part (D2) of that block, which
-// follows the model update, so the rows pass through ldmatrix once. What is left between two model updates is the
-// margin pass, one trip through the cluster, the 16 steps and the update itself. The update reads its rows from the
-// stage (no second register copy), so a stage is held until its block's update is done, and the ring is three deep.
-// The Gram sums exist three times (block mod 3: a CTA sends those of block b + 1 once it has gamma of block b - 1,
-// when a peer may still be reading those of block b - 1), the margin sums twice.
+// What bounds a block. On this part a warp issues one mma.m16n8k16 about every 25 to 30 cycles whatever the number of
+// independent accumulators (the tensor pipe itself is busy 8 cycles per step), so the 48 steps of a warp's pass take
+// 1100 to 1350 cycles and only more warps would shorten them; with eight math warps, the recurrence warp and the copy
+// warp the register file (allocated four warps at a time: 384 threads x 168 registers) has no room for more warps of
+// this size. Measured on one chain of d = 4096 (cycles per block; this kernel: 3860):
+//   - Gram part (D0, D1) of block b + 1 formed while the recurrence warp works on block b, operand registers kept for
+//     the margin part: 3990. The 16 dependent margin steps alone take 750 to 1000 cycles, the recurrence warp's few
+//     loads queue behind eight warps' operand loads in the shared-memory pipe (its sums: 975 cycles instead of 100), and
+//     with the operand registers kept the update has to read its rows from shared memory again (850 instead of 400).
+//   - Margins in fp32 from the row registers (no bf16 copy of the model), Gram part two blocks ahead: 4390 to 4620. The
+//     rows are then unpacked twice per block on the integer pipe, and update and margin pass take 1200 cycles each.
+//   - Gram part by two warps of their own (they fit the register file for free): 4620. One warp needs 4200 cycles for the
+//     128 steps of half the columns, longer than a block.
 //
 // The recurrence warp runs the 16 steps as two groups of 8: within a group every lane steps redundantly on registers (no
 // shuffle in the dependent chain, as in the 8-sample kernels); between the groups the 8 x 8 cross block is applied one
@@ -34,26 +40,24 @@ namespace wpsgd {
 
 constexpr int M16_B = 16;
 constexpr int M16_PAIRS = M16_B * (M16_B - 1) / 2;  // 120
-constexpr int M16_SLOT_FLOATS = 256;   // a warp's table: D0 [16][8] | D1 rows 8..15 [8][8] | p parts [16][4]
-constexpr int M16_GRAM_FLOATS = 192;   // the Gram part of a table
-constexpr int M16_MARGIN_FLOATS = 64;  // the margin part
+constexpr int M16_SLOT_FLOATS = 256;   // D0 [16][8] | D1 rows 8..15 [8][8] | p parts [16][4]
+constexpr uint32_t M16_SLOT_BYTES = M16_SLOT_FLOATS * sizeof(float);
+constexpr int M16_SLOTS = 8;           // one slot per CTA of the cluster
 constexpr int M16_WARPS = 8;           // math warps of a CTA
 
 struct Mma16Smem {
-  size_t row_stride, ring, w3, gred, pred, part, tot, gam, tab, bars, gbar, pbar, flag, total;
-  __host__ __device__ Mma16Smem(int stages, size_t slice_bytes, int cluster) {
+  size_t row_stride, ring, w3, red, part, tot, gam, tab, bars, pbar, flag, total;
+  __host__ __device__ Mma16Smem(int stages, size_t slice_bytes) {
     row_stride = slice_bytes + 16;
     ring = 0;
-    w3 = ring + (size_t)stages * M16_B * row_stride;                       // w_hi, w_mid, w_lo, one zero row
-    gred = w3 + 4 * row_stride;                                            // [3][cluster][192] Gram sums of every CTA
-    pred = gred + 3 * (size_t)cluster * M16_GRAM_FLOATS * sizeof(float);   // [2][cluster][64] margin sums of every CTA
-    part = pred + 2 * (size_t)cluster * M16_MARGIN_FLOATS * sizeof(float); // [math warps][256] this CTA's tables
-    tot = part + (size_t)M16_WARPS * M16_SLOT_FLOATS * sizeof(float);      // [192] Gram sums over the cluster
-    gam = tot + M16_GRAM_FLOATS * sizeof(float);                           // gamma_0..15, 1 - a^nv, stop
-    tab = gam + 32 * sizeof(float);                                        // [3][32]
-    bars = tab + 3 * 32 * sizeof(float);                                   // ring barriers [8]
-    gbar = bars + 8 * sizeof(unsigned long long);                          // Gram-sum barriers [3]
-    pbar = gbar + 4 * sizeof(unsigned long long);                          // margin-sum barriers [2]
+    w3 = ring + (size_t)stages * M16_B * row_stride;                 // w_hi, w_mid, w_lo, one zero row
+    red = w3 + 4 * row_stride;                                       // [2][slots][256] partial sums
+    part = red + 2 * (size_t)M16_SLOTS * M16_SLOT_FLOATS * sizeof(float);  // [math warps][256] this CTA's partial sums
+    tot = part + (size_t)M16_WARPS * M16_SLOT_FLOATS * sizeof(float);      // [256] sums over the slots
+    gam = tot + M16_SLOT_FLOATS * sizeof(float);                     // gamma_0..15, 1 - a^nv, stop
+    tab = gam + 32 * sizeof(float);                                  // [3][32]
+    bars = tab + 3 * 32 * sizeof(float);                             // ring barriers [8]
+    pbar = bars + 8 * sizeof(unsigned long long);                    // partial-sum barriers [2]
     flag = pbar + 2 * sizeof(unsigned long long);
     total = flag + 16;
   }
@@ -90,18 +94,16 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   const int my_chunks = (int)(chunk_end > chunk0 ? chunk_end - chunk0 : 0);
   const size_t slice_bytes = (size_t)cp.chunks_per_cta * 16;
   const size_t ld_bytes = (size_t)p.ld * 2;
-  const Mma16Smem L(S, slice_bytes, (int)C);
+  const Mma16Smem L(S, slice_bytes);
   const size_t row_stride = L.row_stride;
   unsigned char* ring = smem + L.ring;
   unsigned char* w3 = smem + L.w3;
-  float* gred = (float*)(smem + L.gred);
-  float* pred = (float*)(smem + L.pred);
+  float* red = (float*)(smem + L.red);
   float* part = (float*)(smem + L.part);
   float* tot = (float*)(smem + L.tot);
   float* gam = (float*)(smem + L.gam);   // [0..15] gamma, [16] = 1 - a^nv, [17] = leave after this block
   float* tab = (float*)(smem + L.tab);   // [0..16] a^k, [32..48] eta / a^{k+1}, [64..80] 1 - a^k
   unsigned long long* bars = (unsigned long long*)(smem + L.bars);
-  unsigned long long* gbar = (unsigned long long*)(smem + L.gbar);
   unsigned long long* pbar = (unsigned long long*)(smem + L.pbar);
   volatile int* give_up = (volatile int*)(smem + L.flag);
   const char* shard = (const char*)p.X + (size_t)p.shard_off[j] * ld_bytes + (size_t)chunk0 * 16;
@@ -109,7 +111,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   const uint32_t* idx = p.idx + p.idx_off[j];  // padded to a multiple of 64 entries, all valid rows
   const long long nb = (n_run + B - 1) / B;
   const int consumed_threads = (math_warps + 1) * 32;  // math warps arrive, the copy warp waits: named barrier 2
-  const int math_threads = math_warps * 32;
 
   // ---- set-up: tables, barriers, zeroed ring / model rows / partial-sum tables ------------------------------------
   if (threadIdx.x <= B) {  // power tables in fp64, rounded once
@@ -122,7 +123,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   }
   if (threadIdx.x == 32) {
     for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
-    for (int i = 0; i < 3; ++i) mbar_init(&gbar[i], 1);
     mbar_init(&pbar[0], 1);
     mbar_init(&pbar[1], 1);
     *give_up = 0;
@@ -144,69 +144,15 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
     uint32_t id_nxt = 0u;
     if (nb > 0) y_nxt = yshard[idx[n]];
     if (nb > 1) id_nxt = idx[B + n];
+    const uint32_t expect_bytes = C * M16_SLOT_BYTES;
     const bool decaying = p.sched == LR_INV_SQRT;
     const long long first_j = p.first ? p.first[j] : 0;
-    // bounded wait for sums of the whole cluster; a wait that runs out is flagged in every CTA of the cluster
-    auto wait_sums = [&](unsigned long long* bar, uint32_t parity, int where) __attribute__((always_inline)) {
-      bool landed = false;
-      for (long long i = 0; i < bp.spin_limit; ++i) {
-        if (mbar_try_wait_cluster(bar, parity)) { landed = true; break; }
-        if (*give_up) break;
-      }
-      if (!landed && !*give_up) {
-        set_status(p.status, DEV_TIMEOUT, where, (long long)blockIdx.x);
-        for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
-      }
-    };
-    // The Gram entries of a block, into registers: Gaa, Gbb the strict lower triangles of the two 8 x 8 diagonal blocks
-    // (the same in every lane), gba this lane's row of the cross block. Runs while the math warps are busy with the
-    // update and the margin pass of the block before.
-    float Gaa[BLK_PAIRS], Gbb[BLK_PAIRS], gba[8];
-    auto take_gram = [&](long long b) __attribute__((always_inline)) {
-      const int q3 = (int)(b % 3);
-      if (lane == 0) mbar_arrive_expect_tx(&gbar[q3], C * (uint32_t)(M16_GRAM_FLOATS * sizeof(float)));
-      wait_sums(&gbar[q3], (uint32_t)((b / 3) & 1), 3);
-      if (lane < M16_GRAM_FLOATS / 8) {  // lane l adds the 16-byte groups l and l + 24 over the CTAs, in rank order
-        const float4* r4 = (const float4*)(gred + (size_t)q3 * C * M16_GRAM_FLOATS);
-        float4 s0 = r4[lane], s1 = r4[24 + lane];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) {
-          if ((uint32_t)w >= C) break;
-          const float4 v0 = r4[w * (M16_GRAM_FLOATS / 4) + lane], v1 = r4[w * (M16_GRAM_FLOATS / 4) + 24 + lane];
-          s0.x += v0.x; s0.y += v0.y; s0.z += v0.z; s0.w += v0.w;
-          s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
-        }
-        ((float4*)tot)[lane] = s0;
-        ((float4*)tot)[24 + lane] = s1;
-      }
-      __syncwarp();
-#pragma unroll
-      for (int n2 = 1; n2 < 8; ++n2) {
-        const float4 lo = *(const float4*)&tot[n2 * 8], hi = *(const float4*)&tot[n2 * 8 + 4];
-        const float row[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          if (k < n2) Gaa[n2 * (n2 - 1) / 2 + k] = row[k];
-        const float4 lo2 = *(const float4*)&tot[128 + n2 * 8], hi2 = *(const float4*)&tot[128 + n2 * 8 + 4];
-        const float row2[8] = {lo2.x, lo2.y, lo2.z, lo2.w, hi2.x, hi2.y, hi2.z, hi2.w};
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          if (k < n2) Gbb[n2 * (n2 - 1) / 2 + k] = row2[k];
-      }
-      {
-        const int own = 8 + (lane & 7);  // this lane's sample of group B
-        const float4 lo = *(const float4*)&tot[own * 8], hi = *(const float4*)&tot[own * 8 + 4];
-        gba[0] = lo.x; gba[1] = lo.y; gba[2] = lo.z; gba[3] = lo.w; gba[4] = hi.x; gba[5] = hi.y; gba[6] = hi.z; gba[7] = hi.w;
-      }
-      __syncwarp();  // tot is read; the next block may overwrite it
-    };
     cluster_barrier();  // start-up: every CTA of the cluster runs and has set up its shared memory
-    if (nb > 0) take_gram(0);
 
     for (long long b = 0; b < nb; ++b) {
       const int nv = (int)((n_run - b * B) < (long long)B ? (n_run - b * B) : (long long)B);
       const int q = (int)(b & 1);
-      if (lane == 0) mbar_arrive_expect_tx(&pbar[q], C * (uint32_t)(M16_MARGIN_FLOATS * sizeof(float)));
+      if (lane == 0) mbar_arrive_expect_tx(&pbar[q], expect_bytes);
       const float y_cur = y_nxt;  // lane l: label of sample l & 15
       if (b + 1 < nb) y_nxt = yshard[id_nxt];
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
@@ -218,6 +164,35 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       } else {
 #pragma unroll
         for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[32 + m]; }
+      }
+      // ---- wait (bounded) for the partial sums of block b from every math warp of the cluster ------------------
+      {
+        const uint32_t parity = (uint32_t)((b >> 1) & 1);
+        bool landed = false;
+        for (long long i = 0; i < bp.spin_limit; ++i) {
+          if (mbar_try_wait_cluster(&pbar[q], parity)) { landed = true; break; }
+          if (*give_up) break;
+        }
+        if (!landed && !*give_up) {
+          set_status(p.status, DEV_TIMEOUT, 2, (long long)blockIdx.x);
+          for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
+        }
+      }
+      const int stop = *give_up;
+      // ---- sum over the slots: lane l adds the 16-byte groups l and l + 32 of every slot ---------------------------
+      {
+        const float4* r4 = (const float4*)(red + (size_t)q * M16_SLOTS * M16_SLOT_FLOATS);
+        float4 s0 = r4[lane], s1 = r4[32 + lane];
+#pragma unroll
+        for (int w = 1; w < M16_SLOTS; ++w) {
+          if ((uint32_t)w >= C) break;
+          const float4 v0 = r4[w * (M16_SLOT_FLOATS / 4) + lane], v1 = r4[w * (M16_SLOT_FLOATS / 4) + 32 + lane];
+          s0.x += v0.x; s0.y += v0.y; s0.z += v0.z; s0.w += v0.w;
+          s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
+        }
+        ((float4*)tot)[lane] = s0;
+        ((float4*)tot)[32 + lane] = s1;
+        __syncwarp();
       }
       // ---- the 16 steps as two groups of 8 (samples A = 0..7, B = 8..15). Within a group every lane runs the steps
       // redundantly on registers (28 Gram entries, no shuffle in the dependent chain); between the groups lane l forms
@@ -237,35 +212,36 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
         }
         if (m >= nv) cf[m] = 0.0f;  // samples beyond the chain's end take no step
       }
-      // ---- the margins of block b from every CTA of the cluster (bounded wait), added in rank order ----------------
-      wait_sums(&pbar[q], (uint32_t)((b >> 1) & 1), 2);
-      const int stop = *give_up;
+      float Gaa[BLK_PAIRS], Gbb[BLK_PAIRS], gba[8];
+#pragma unroll
+      for (int n2 = 1; n2 < 8; ++n2) {
+        const float4 lo = *(const float4*)&tot[n2 * 8], hi = *(const float4*)&tot[n2 * 8 + 4];
+        const float row[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (k < n2) Gaa[n2 * (n2 - 1) / 2 + k] = row[k];
+        const float4 lo2 = *(const float4*)&tot[128 + n2 * 8], hi2 = *(const float4*)&tot[128 + n2 * 8 + 4];
+        const float row2[8] = {lo2.x, lo2.y, lo2.z, lo2.w, hi2.x, hi2.y, hi2.z, hi2.w};
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (k < n2) Gbb[n2 * (n2 - 1) / 2 + k] = row2[k];
+      }
       {
-        const float4* p4 = (const float4*)(pred + (size_t)q * C * M16_MARGIN_FLOATS);
+        const int own = 8 + (lane & 7);  // this lane's sample of group B
+        const float4 lo = *(const float4*)&tot[own * 8], hi = *(const float4*)&tot[own * 8 + 4];
+        gba[0] = lo.x; gba[1] = lo.y; gba[2] = lo.z; gba[3] = lo.w; gba[4] = hi.x; gba[5] = hi.y; gba[6] = hi.z; gba[7] = hi.w;
+      }
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          float4 pp = p4[m];  // w_hi . x, w_mid . x, w_lo . x; small terms first
-#pragma unroll
-          for (int w = 1; w < 8; ++w) {
-            if ((uint32_t)w >= C) break;
-            const float4 v = p4[w * (M16_MARGIN_FLOATS / 4) + m];
-            pp.x += v.x; pp.y += v.y; pp.z += v.z;
-          }
-          r[m] = (pp.z + pp.y) + pp.x;
-        }
+      for (int m = 0; m < 8; ++m) {
+        const float4 pp = *(const float4*)&tot[192 + 4 * m];  // w_hi . x, w_mid . x, w_lo . x; small terms first
+        r[m] = (pp.z + pp.y) + pp.x;
       }
       float r_own;
       {
-        const float4* p4 = (const float4*)(pred + (size_t)q * C * M16_MARGIN_FLOATS) + 8 + (lane & 7);
-        float4 pp = p4[0];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) {
-          if ((uint32_t)w >= C) break;
-          const float4 v = p4[w * (M16_MARGIN_FLOATS / 4)];
-          pp.x += v.x; pp.y += v.y; pp.z += v.z;
-        }
+        const float4 pp = *(const float4*)&tot[192 + 4 * (8 + (lane & 7))];
         r_own = (pp.z + pp.y) + pp.x;
       }
+      __syncwarp();  // tot is read; the next block may overwrite it
       float mine = dl_nv;  // lane 16 publishes 1 - a^nv
 #pragma unroll
       for (int m = 0; m < 8; ++m) {  // group A
@@ -293,7 +269,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       if (lane <= B + 1) gam[lane] = mine;
       __syncthreads();  // gamma and the decision published
       if (stop) break;
-      if (b + 1 < nb) take_gram(b + 1);
     }
     cluster_barrier();  // nobody exits while a peer may still store into its shared memory
     return;
@@ -302,9 +277,9 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   if (warp == 1) {
     // =========================== copy warp ==============================================================
     // Lane m < 16 requests this CTA's column slice of row m of a block as one bulk copy; the sixteen copies complete
-    // on the stage's barrier. A stage is refilled as soon as every math warp of this CTA has applied the block's update
-    // from it (they arrive on a named barrier that this warp waits on); with a ring of three the rows of a block have
-    // two block times to arrive.
+    // on the stage's barrier. A stage is refilled as soon as every math warp of this CTA has run its tensor-core passes
+    // over it and holds its own columns of the rows in registers (they arrive on a named barrier that this warp waits
+    // on): well before the block's gamma is known, so the rows of block b + 2 have a whole block time to arrive.
     const uint32_t copy_bytes = (uint32_t)my_chunks * 16u;
     uint32_t id_next = 0u;
     auto peek = [&](long long blk) {
@@ -330,13 +305,13 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
     long long b = 0;
     bool stop = false;
     for (; b < nb; ++b) {
-      __syncthreads();  // gamma_b and the decision
-      if (gam[B + 1] != 0.0f) { stop = true; break; }
-      asm volatile("bar.sync 2, %0;" ::"r"(consumed_threads) : "memory");  // the update of block b has read its stage
+      asm volatile("bar.sync 2, %0;" ::"r"(consumed_threads) : "memory");  // the stage of block b has been read
       request(requested, st);
       ++requested;
       peek(requested);
       st = (st + 1 == S) ? 0 : st + 1;
+      __syncthreads();
+      if (gam[B + 1] != 0.0f) { stop = true; ++b; break; }
     }
     if (stop && copy_bytes > 0) {
       // leave no copy in flight into this CTA's shared memory: wait (bounded) on the stage of every block that was
@@ -406,15 +381,60 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       for (uint32_t rr = 0; rr < C; ++rr) st_shared_cluster(map_shared_rank((const void*)give_up, rr), 1);
     }
   };
-  const int mt = mw * 32 + lane;
-  uint32_t xk[16][4];  // the A tiles of a block's rows over this warp's columns: loaded by the Gram pass, kept for the margin pass
-  // adds the math warps' tables up over the 16-byte groups [g0, g0 + n) in warp order and sends the sums to this CTA's
-  // place in every CTA of the cluster (after a barrier among the math warps: the tables are written)
-  auto reduce_and_send = [&](int g0, int n, float* dst, unsigned long long* bar) __attribute__((always_inline)) {
-    asm volatile("bar.sync 3, %0;" ::"r"(math_threads) : "memory");
-    const uint32_t ob = (uint32_t)__cvta_generic_to_shared(bar) - own_base;
-    for (int e = mt; e < n; e += math_threads) {
-      const float4* p4 = (const float4*)part + g0 + e;
+  // D0, D1, D2 of a block over this warp's columns, sent to this warp's slot of every CTA of the cluster
+  auto tensor_pass = [&](const unsigned char* stage, int q, uint4 (&raw)[B]) __attribute__((always_inline)) {
+    float d0[2][4], d1[2][4], d2[2][4];  // two independent accumulator sets (a dependent mma takes about 20 cycles)
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) d0[a][e] = d1[a][e] = d2[a][e] = 0.0f;
+    const unsigned char* xs = stage + x_off;
+#pragma unroll
+    for (int round = 0; round < 8; ++round) {
+      uint32_t xa[2][4], wb[2][2];
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+        if (round * 2 + a < ksteps) {
+          ldmatrix_x4(xa[a], xs + (size_t)(round * 2 + a) * 32);
+          ldmatrix_x2(wb[a], w_src + (size_t)(round * 2 + a) * 32);
+        }
+      // this thread's columns of two of the 16 rows, for the update: between the tensor-core steps these loads find the
+      // shared-memory pipe idle; after the pass they would queue ahead of the sums that the recurrence warp waits for
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        const int m = round * 2 + a;
+        raw[m] = act ? *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+        if (round * 2 + a < ksteps) {
+          mma_bf16_m16n8k16(d0[a], xa[a][0], xa[a][1], xa[a][2], xa[a][3], xa[a][0], xa[a][2]);
+          mma_bf16_m16n8k16(d1[a], xa[a][0], xa[a][1], xa[a][2], xa[a][3], xa[a][1], xa[a][3]);
+          mma_bf16_m16n8k16(d2[a], xa[a][0], xa[a][1], xa[a][2], xa[a][3], wb[a][0], wb[a][1]);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      d0[0][e] += d0[1][e];
+      d1[0][e] += d1[1][e];
+      d2[0][e] += d2[1][e];
+    }
+    asm volatile("bar.arrive 2, %0;" ::"r"(consumed_threads) : "memory");  // this warp is done with the stage of the block
+    // Two-level sum. Each warp puts its accumulators (row g8 / g8 + 8, columns 2 t4, 2 t4 + 1) into its own table of
+    // this CTA; after a barrier among the math warps the first 64 math threads add the tables up in a fixed order,
+    // 16 bytes each, and send the CTA's sums to this CTA's slot in every CTA of the cluster.
+    float* sl = part + (size_t)mw * M16_SLOT_FLOATS;
+    *(float2*)(sl + g8 * 8 + 2 * t4) = make_float2(d0[0][0], d0[0][1]);
+    *(float2*)(sl + (g8 + 8) * 8 + 2 * t4) = make_float2(d0[0][2], d0[0][3]);
+    *(float2*)(sl + 128 + g8 * 8 + 2 * t4) = make_float2(d1[0][2], d1[0][3]);
+    if (t4 < 2) {  // columns 0..3 of D2: the three parts of p and the zero row
+      *(float2*)(sl + 192 + g8 * 4 + 2 * t4) = make_float2(d2[0][0], d2[0][1]);
+      *(float2*)(sl + 192 + (g8 + 8) * 4 + 2 * t4) = make_float2(d2[0][2], d2[0][3]);
+    }
+    asm volatile("bar.sync 3, %0;" ::"r"(math_warps * 32) : "memory");
+    const uint32_t ob = (uint32_t)__cvta_generic_to_shared(&pbar[q]) - own_base;
+    for (int e = mw * 32 + lane; e < M16_SLOT_FLOATS / 4; e += math_warps * 32) {
+      const float4* p4 = (const float4*)part + e;
       float4 sum = p4[0];
 #pragma unroll
       for (int w = 1; w < M16_WARPS; ++w)
@@ -422,77 +442,22 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
           const float4 v = p4[w * (M16_SLOT_FLOATS / 4)];
           sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
-      const uint32_t od = (uint32_t)__cvta_generic_to_shared(dst + 4 * e) - own_base;
+      const uint32_t od = (uint32_t)__cvta_generic_to_shared(red + ((size_t)q * M16_SLOTS + rank) * M16_SLOT_FLOATS + 4 * e) - own_base;
 #pragma unroll
       for (int rr = 0; rr < 8; ++rr)
         if ((uint32_t)rr < C) st_async_f32x4(peer_base[rr] + od, sum, peer_base[rr] + ob);
     }
   };
-  // D0, D1 of a block over this warp's columns (accumulator: rows g8 / g8 + 8, columns 2 t4, 2 t4 + 1)
-  auto gram_pass = [&](const unsigned char* stage, long long blk) __attribute__((always_inline)) {
-    float d0[2][4], d1[2][4];  // two independent accumulator sets (a dependent mma takes about 20 cycles)
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) d0[a][e] = d1[a][e] = 0.0f;
-    const unsigned char* xs = stage + x_off;
-#pragma unroll
-    for (int ks = 0; ks < 16; ++ks)
-      if (ks < ksteps) {
-        ldmatrix_x4(xk[ks], xs + (size_t)ks * 32);
-        mma_bf16_m16n8k16(d0[ks & 1], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3], xk[ks][0], xk[ks][2]);
-        mma_bf16_m16n8k16(d1[ks & 1], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3], xk[ks][1], xk[ks][3]);
-      }
-    float* sl = part + (size_t)mw * M16_SLOT_FLOATS;
-    *(float2*)(sl + g8 * 8 + 2 * t4) = make_float2(d0[0][0] + d0[1][0], d0[0][1] + d0[1][1]);
-    *(float2*)(sl + (g8 + 8) * 8 + 2 * t4) = make_float2(d0[0][2] + d0[1][2], d0[0][3] + d0[1][3]);
-    *(float2*)(sl + 128 + g8 * 8 + 2 * t4) = make_float2(d1[0][2] + d1[1][2], d1[0][3] + d1[1][3]);
-    const int q3 = (int)(blk % 3);
-    reduce_and_send(0, M16_GRAM_FLOATS / 4, gred + ((size_t)q3 * C + rank) * M16_GRAM_FLOATS, &gbar[q3]);
-  };
-  // D2 of the block whose A tiles are in xk, with the model as it stands
-  auto margin_pass = [&](int q) __attribute__((always_inline)) {
-    float d2[2][4];
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) d2[a][e] = 0.0f;
-#pragma unroll
-    for (int ks = 0; ks < 16; ++ks)
-      if (ks < ksteps) {
-        uint32_t wb[2];
-        ldmatrix_x2(wb, w_src + (size_t)ks * 32);
-        mma_bf16_m16n8k16(d2[ks & 1], xk[ks][0], xk[ks][1], xk[ks][2], xk[ks][3], wb[0], wb[1]);
-      }
-    if (t4 < 2) {  // columns 0..3 of D2: the three parts of p and the zero row
-      float* sl = part + (size_t)mw * M16_SLOT_FLOATS + M16_GRAM_FLOATS;
-      *(float2*)(sl + g8 * 4 + 2 * t4) = make_float2(d2[0][0] + d2[1][0], d2[0][1] + d2[1][1]);
-      *(float2*)(sl + (g8 + 8) * 4 + 2 * t4) = make_float2(d2[0][2] + d2[1][2], d2[0][3] + d2[1][3]);
-    }
-    reduce_and_send(M16_GRAM_FLOATS / 4, M16_MARGIN_FLOATS / 4, pred + ((size_t)q * C + rank) * M16_MARGIN_FLOATS, &pbar[q]);
-  };
 
   int st = 0;
   uint32_t par = 0u;
-  if (nb > 0) {
-    wait_rows(0, 0u);
-    gram_pass(ring, 0);
-  }
   for (long long b = 0; b < nb; ++b) {
+    wait_rows(st, par);
     const unsigned char* stage = ring + (size_t)st * B * row_stride;
-    margin_pass((int)(b & 1));
-    if (b + 1 < nb) {  // the Gram part of the next block, while the recurrence warp works on this one
-      const int st1 = (st + 1 == S) ? 0 : st + 1;
-      wait_rows(st1, (st + 1 == S) ? (par ^ 1u) : par);
-      gram_pass(ring + (size_t)st1 * B * row_stride, b + 1);
-    }
-    __syncthreads();  // gamma_b and the decision are in gam
-    if (gam[B + 1] != 0.0f) {
-      // giving up: sums sent just now may still be on their way to a peer; let them land before anyone exits
-      const long long t0 = clock64();
-      while (clock64() - t0 < 100000) {}
-      break;
-    }
+    uint4 raw[B];  // this thread's columns of the 16 rows, for the update
+    tensor_pass(stage, (int)(b & 1), raw);
+    __syncthreads();  // gamma_b and the decision are in gam; every math warp is done with the stage of block b
+    if (gam[B + 1] != 0.0f) break;
     // ---- w <- w - (1 - a^nv) w - sum_m gamma_m x_m, then the model rows again -----------------------------------------
     if (act) {
       const float ndl = -gam[B];
@@ -504,8 +469,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       for (int m = 0; m < B; ++m) {
         const float gm = -gam[m];
         const float2 g2 = make_float2(gm, gm);
-        const uint4 raw = *(const uint4*)(stage + (size_t)m * row_stride + (size_t)lc * 16);
-        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+        const uint32_t rw[4] = {raw[m].x, raw[m].y, raw[m].z, raw[m].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           wv[i] = __ffma2_rn(g2, make_float2(__uint_as_float(rw[i] << 16), __uint_as_float(rw[i] & 0xffff0000u)), wv[i]);
@@ -513,7 +477,6 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
 #pragma unroll
       for (int i = 0; i < 4; ++i) w2[i] = wv[i];
     }
-    asm volatile("bar.arrive 2, %0;" ::"r"(consumed_threads) : "memory");  // this warp is done with the stage of block b
     publish_model();
     if (++st == S) { st = 0; par ^= 1u; }
   }

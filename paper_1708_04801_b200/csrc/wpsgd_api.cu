@@ -322,7 +322,6 @@ wpsgd_status launch_reg_pf(wpsgd_ctx* c, const ChainParams& p, bool bpn, int thr
 
 // ---- blocked chain kernel: shapes it takes, ring depth, launch ------------------------------------------------
 constexpr size_t kSmemBudget = 220 * 1024;
-constexpr size_t kSmemMax = 227 * 1024;  // the most dynamic shared memory a CTA can have
 
 template <typename XT>
 bool block_kernel_fits(const wpsgd_ctx* c, bool aligned, int* threads_out, int* R_out, int* stages_out) {
@@ -434,9 +433,8 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   out->math_warps = (int)mw;
   out->stages = stages;
   // 16 samples per block (squared and hinge losses): half as many hand-offs per sample; one CTA per SM
-  // (a stage is held until its block's update is done while the next block's Gram pass already reads its own: three deep)
-  int s16 = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 3;
-  while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16, C).total > kSmemMax) --s16;
+  int s16 = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
+  while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16).total > kSmemBudget) --s16;
   out->stages16 = s16 >= 2 ? s16 : 0;
   const bool can16 = out->stages16 > 0 && c->loss != WPSGD_LOSS_LOGISTIC;
   out->block = (c->opt_block_samples == 16 || (c->opt_block_samples == 0 && can16)) ? 16 : 8;
@@ -455,7 +453,7 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   cp.chunks_per_cta = sh.cpc;
   const bool b16 = sh.block == 16;
   if (b16) cp.b.stages = sh.stages16;
-  const size_t smem = b16 ? Mma16Smem(sh.stages16, (size_t)sh.cpc * 16, sh.C).total : MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
+  const size_t smem = b16 ? Mma16Smem(sh.stages16, (size_t)sh.cpc * 16).total : MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
