@@ -356,8 +356,10 @@ def measure(P, multi, wl, cfg, dev, steps, warmup, peak, peak_src, options, worl
             "traffic": None, "peak_source": f"of {peak_src}", "kernel": "chain kernel (per-node SGD loops)",
             "kernel_ms": chain_med, "kernel_ms_best": chain_best, "algorithmic_bytes_per_launch": alg_bytes,
             "bytes_per_sample_update": bytes_per_update(wl),
-            # what a chain-per-resource schedule can reach at best, and how much of the GPU the launch covers
-            "node_pinned_ceiling": float(wl.total_steps) / float(wl.k * max(longest, 1)),
+            # mean chain length over the longest: the busy share of a schedule that gives every chain its own SMs for
+            # the whole launch (chains that take turns on the same SMs, as the cluster kernels' do, can exceed it);
+            # and how much of the GPU the launch covers
+            "mean_over_longest_chain": float(wl.total_steps) / float(wl.k * max(longest, 1)),
             "ctas": ctas, "sm_coverage": min(1.0, ctas / N_SMS),
             # the serial side of the same kernel: device cycles per sample-update of the longest chain
             "cycles_per_update_longest_chain": chain_med * 1e-3 * mhz * 1e6 / max(longest, 1)}

@@ -27,6 +27,8 @@
 //     rows are then unpacked twice per block on the integer pipe, and update and margin pass take 1200 cycles each.
 //   - Gram part by two warps of their own (they fit the register file for free): 4620. One warp needs 4200 cycles for the
 //     128 steps of half the columns, longer than a block.
+//   - Ten math warps of 26 chunks instead of eight of 32 (the register allocation is the same): 4560.
+//   - gamma of the first eight samples handed to the math warps while the other eight steps run: 3890 (no gain).
 //
 // The recurrence warp runs the 16 steps as two groups of 8: within a group every lane steps redundantly on registers (no
 // shuffle in the dependent chain, as in the 8-sample kernels); between the groups the 8 x 8 cross block is applied one
