@@ -45,10 +45,10 @@ N_SMS = 148
 # DRAM bytes (read + write) per launch of the chain kernel from an ncu capture, with the hash of the
 # kernel sources the capture was taken from; reported as null once the sources have changed.
 NCU_TRAFFIC = {
-    "config3": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 26349015040,
+    "config3": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 26347168248,
                 "note": "captured with 2048 rows per node (2 GiB on the device): same step counts and kernel work per launch, no scaling"},
-    "config5": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 15945717400, "note": "full-size capture"},
-    "config4": {"src_sha": "364373e1d295c7a1", "bytes_per_launch": 4275997808, "note": "full-size capture"},
+    "config5": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 15944920632, "note": "full-size capture"},
+    "config4": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 4306268816, "note": "full-size capture"},
 }
 
 

@@ -750,7 +750,8 @@ struct BlockWarpSmem {
   }
 };
 
-template <typename XT, int R, int LOSS>
+// DECAY: the step size decays (per-block tables); the constant schedule is compiled without that code
+template <typename XT, int R, int LOSS, bool DECAY>
 __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(const BlockParams bp) {
   constexpr int V = XVec<XT>::V;
   constexpr int QV = V / 4;
@@ -791,8 +792,7 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
   float apw[B], cfac[B];
 #pragma unroll
   for (int m = 0; m < B; ++m) { apw[m] = tab[m]; cfac[m] = tab[16 + m]; }
-  const bool decaying = p.sched == LR_INV_SQRT;
-  const long long first_j = p.first ? p.first[j] : 0;
+  const long long first_j = (DECAY && p.first) ? p.first[j] : 0;
 
   bool act[R];
   float w[R][V];
@@ -917,7 +917,7 @@ __global__ void __launch_bounds__(32 * BLKW_MAX_WARPS) chain_block_warp_kernel(c
     __syncwarp();
     // ---- 8-step recurrence, every lane the same ----------------------------------------------------------
     float a_nv = tab[nv], dl = tab[32 + nv], apw_own = tab[n];
-    if (decaying) decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl);
+    if (DECAY) decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl);
     float t[B], beta[B], yv[B], cf[B], sc[B];
 #pragma unroll
     for (int m = 0; m < B; ++m) yv[m] = __shfl_sync(0xffffffffu, y_cur, m);

@@ -560,10 +560,11 @@ wpsgd_status launch_block_warp_r(wpsgd_ctx* c, const BlockParams& bp, size_t sme
     c->launches++;
     return WPSGD_OK;
   };
+  const bool decay = c->sched == WPSGD_LR_INV_SQRT;
   switch (c->loss) {
-    case WPSGD_LOSS_HINGE: return go(chain_block_warp_kernel<XT, R, LOSS_HINGE>);
-    case WPSGD_LOSS_LOGISTIC: return go(chain_block_warp_kernel<XT, R, LOSS_LOGISTIC>);
-    default: return go(chain_block_warp_kernel<XT, R, LOSS_SQUARED>);
+    case WPSGD_LOSS_HINGE: return decay ? go(chain_block_warp_kernel<XT, R, LOSS_HINGE, true>) : go(chain_block_warp_kernel<XT, R, LOSS_HINGE, false>);
+    case WPSGD_LOSS_LOGISTIC: return decay ? go(chain_block_warp_kernel<XT, R, LOSS_LOGISTIC, true>) : go(chain_block_warp_kernel<XT, R, LOSS_LOGISTIC, false>);
+    default: return decay ? go(chain_block_warp_kernel<XT, R, LOSS_SQUARED, true>) : go(chain_block_warp_kernel<XT, R, LOSS_SQUARED, false>);
   }
 }
 
