@@ -367,7 +367,8 @@ def measure(P, multi, wl, cfg, dev, steps, warmup, peak, peak_src, options, worl
     roof["limiter"] = ("chain latency: the longest chain's dependent steps, not a memory level"
                        if (roof["frac"] < 0.2 or ctas < N_SMS) else "dependent loop of a block and HBM together (see the profile)")
     tr = NCU_TRAFFIC.get(f"config{cfg}", {})
-    if tr.get("src_sha") == kernel_src_sha() and not small:
+    # (config 5 was captured at speed ratio 4: the workload's name carries the ratio)
+    if tr.get("src_sha") == kernel_src_sha() and not small and (cfg != 5 or wl.name == "config5_rho4"):
         roof["traffic"] = tr.get("bytes_per_launch")
         roof["traffic_note"] = tr.get("note")
     entry = {"workload": describe(wl, cfg, small), "value": float(wl.total_steps) * world * steps / (total_ms * 1e-3),
