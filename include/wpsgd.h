@@ -90,8 +90,7 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
  *   "sparse_variant"  kernel for CSR rows. 0 (default) and 2: blocks of up to 64 steps run in a shared-memory cache of
  *                     the model entries they touch. 1: one step per round trip to the model in global memory.
  *   "cluster"         CTAs per node of variant 8: 0 (default) chosen from d, else 1, 2, 4 or 8.
- *   "block_samples"   samples per block of variant 8: 0 (default) 16 for the squared and hinge losses when the rows
- *                     fit, else 8; 8 or 16 to force one (16 with the logistic loss: WPSGD_ERR_UNSUPPORTED).
+ *   "block_samples"   samples per block of variant 8: 0 (default) 16 when the rows fit, else 8; 8 or 16 to force one.
  *   "threads"         threads per node of variants 2 and 4, warps x 32 per CTA of variant 5; 0 (default): chosen from d.
  *   "prefetch"        rows in flight per chain of variants 2, 3 and of sparse variant 1; 0 (default): chosen.
  *   "stages"          blocks of rows in the shared-memory ring of the blocked kernels; 0 (default): as many as fit

@@ -32,8 +32,8 @@
 //
 // The recurrence warp runs the 16 steps as two groups of 8: within a group every lane steps redundantly on registers (no
 // shuffle in the dependent chain, as in the 8-sample kernels); between the groups the 8 x 8 cross block is applied one
-// row per lane and gathered with eight shuffles. Losses: squared and hinge; the logistic loss stays with the 8-sample
-// kernels.
+// row per lane and gathered with eight shuffles. The logistic loss runs each group through the 8-sample recurrence with
+// its factor expanded around the group's margins (block8_recurrence).
 #pragma once
 
 #include "chain_mma.cuh"
@@ -48,7 +48,7 @@ constexpr int M16_SLOTS = 8;           // one slot per CTA of the cluster
 constexpr int M16_WARPS = 8;           // math warps of a CTA
 
 struct Mma16Smem {
-  size_t row_stride, ring, w3, red, part, tot, gam, tab, bars, pbar, flag, total;
+  size_t row_stride, ring, w3, red, part, tot, gam, tab, jet, bars, pbar, flag, total;
   __host__ __device__ Mma16Smem(int stages, size_t slice_bytes) {
     row_stride = slice_bytes + 16;
     ring = 0;
@@ -58,7 +58,8 @@ struct Mma16Smem {
     tot = part + (size_t)M16_WARPS * M16_SLOT_FLOATS * sizeof(float);      // [256] sums over the slots
     gam = tot + M16_SLOT_FLOATS * sizeof(float);                     // gamma_0..15, 1 - a^nv, stop
     tab = gam + 32 * sizeof(float);                                  // [3][32]
-    bars = tab + 3 * 32 * sizeof(float);                             // ring barriers [8]
+    jet = tab + 3 * 32 * sizeof(float);                              // 8 x (s, s', s''/2, s'''/6) of the logistic factor
+    bars = jet + 8 * 4 * sizeof(float);                             // ring barriers [8]
     pbar = bars + 8 * sizeof(unsigned long long);                    // partial-sum barriers [2]
     flag = pbar + 2 * sizeof(unsigned long long);
     total = flag + 16;
@@ -104,6 +105,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
   float* part = (float*)(smem + L.part);
   float* tot = (float*)(smem + L.tot);
   float* gam = (float*)(smem + L.gam);   // [0..15] gamma, [16] = 1 - a^nv, [17] = leave after this block
+  float4* jets = (float4*)(smem + L.jet);
   float* tab = (float*)(smem + L.tab);   // [0..16] a^k, [32..48] eta / a^{k+1}, [64..80] 1 - a^k
   unsigned long long* bars = (unsigned long long*)(smem + L.bars);
   unsigned long long* pbar = (unsigned long long*)(smem + L.pbar);
@@ -160,8 +162,8 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
       if (b + 2 < nb) id_nxt = idx[(b + 2) * B + n];
       float a_nv = tab[nv], dl_nv = tab[64 + nv];
       float apw[B], cfac[B];
+      float apw_own = tab[n];  // A of this lane's own sample (lane & 15)
       if (decaying) {
-        float apw_own;
         decaying_block_tables<B>((double)p.eta0, (double)p.lambda, first_j + b * B, nv, apw, cfac, apw_own, a_nv, dl_nv);
       } else {
 #pragma unroll
@@ -205,7 +207,10 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
 #pragma unroll
       for (int m = 0; m < B; ++m) {
         yv[m] = __shfl_sync(0xffffffffu, y_cur, m);
-        if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
+        if (LOSS == LOSS_LOGISTIC) {  // g = -y / (1 + 2^t), t = y a^n log2(e) (...)
+          sc[m] = yv[m] * apw[m] * 1.4426950408889634f;
+          cf[m] = -yv[m] * cfac[m];
+        } else if (LOSS == LOSS_HINGE) {  // g = -y if t < 1, t = y a^n (...)
           sc[m] = yv[m] * apw[m];
           cf[m] = -yv[m] * cfac[m];
         } else {  // squared: g = t - y, t = a^n (...)
@@ -243,8 +248,42 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
         const float4 pp = *(const float4*)&tot[192 + 4 * (8 + (lane & 7))];
         r_own = (pp.z + pp.y) + pp.x;
       }
+      float p_own_a = 0.0f;  // margin of sample lane & 7 (the logistic expansion of group A is formed one sample per lane)
+      if (LOSS == LOSS_LOGISTIC) {
+        const float4 pp = *(const float4*)&tot[192 + 4 * (lane & 7)];
+        p_own_a = (pp.z + pp.y) + pp.x;
+      }
       __syncwarp();  // tot is read; the next block may overwrite it
       float mine = dl_nv;  // lane 16 publishes 1 - a^nv
+      if (LOSS == LOSS_LOGISTIC) {
+        // The same two groups through the 8-sample recurrence with the logistic factor expanded around each group's
+        // margins (see block8_recurrence): arguments and Gram entries scaled by sc_n beforehand.
+        const float sc_own = y_cur * apw_own * 1.4426950408889634f;  // of sample lane & 15
+        const float sc_own_a = __shfl_sync(0xffffffffu, sc_own, lane & 7), sc_own_b = __shfl_sync(0xffffffffu, sc_own, 8 + (lane & 7));
+        float t8[8], cf8[8], yv8[8], b8[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          t8[m] = sc[m] * r[m]; cf8[m] = cf[m]; yv8[m] = yv[m];
+#pragma unroll
+          for (int k2 = 0; k2 < m; ++k2) Gaa[m * (m - 1) / 2 + k2] *= sc[m];
+        }
+        block8_recurrence<LOSS>(t8, Gaa, cf8, yv8, sc_own_a * p_own_a, jets, b8);
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          beta[m] = b8[m];
+          r_own = fmaf(-b8[m], gba[m], r_own);
+        }
+        __syncwarp();  // every lane has read the expansions of group A
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          t8[m] = sc[8 + m] * __shfl_sync(0xffffffffu, r_own, m); cf8[m] = cf[8 + m]; yv8[m] = yv[8 + m];
+#pragma unroll
+          for (int k2 = 0; k2 < m; ++k2) Gbb[m * (m - 1) / 2 + k2] *= sc[8 + m];
+        }
+        block8_recurrence<LOSS>(t8, Gbb, cf8, yv8, sc_own_b * r_own, jets, b8);
+#pragma unroll
+        for (int m = 0; m < 8; ++m) beta[8 + m] = b8[m];
+      } else {
 #pragma unroll
       for (int m = 0; m < 8; ++m) {  // group A
         const float tm_ = sc[m] * r[m];
@@ -263,6 +302,7 @@ __global__ void __launch_bounds__(64 + 32 * 8, 1) chain_mma16_kernel(const Clust
         else beta[8 + m] = cf[8 + m] * (tm_ - yv[8 + m]);
 #pragma unroll
         for (int n2 = m + 1; n2 < 8; ++n2) r[8 + n2] = fmaf(-beta[8 + m], Gbb[n2 * (n2 - 1) / 2 + m], r[8 + n2]);
+      }
       }
 #pragma unroll
       for (int m = 0; m < B; ++m)

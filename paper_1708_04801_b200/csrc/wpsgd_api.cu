@@ -436,7 +436,7 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   int s16 = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
   while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16).total > kSmemBudget) --s16;
   out->stages16 = s16 >= 2 ? s16 : 0;
-  const bool can16 = out->stages16 > 0 && c->loss != WPSGD_LOSS_LOGISTIC;
+  const bool can16 = out->stages16 > 0;
   out->block = (c->opt_block_samples == 16 || (c->opt_block_samples == 0 && can16)) ? 16 : 8;
   if (out->block == 16 && !can16) return false;
   return true;
@@ -472,7 +472,13 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
     c->launches++;
     return WPSGD_OK;
   };
-  if (b16) return c->loss == WPSGD_LOSS_HINGE ? go(chain_mma16_kernel<LOSS_HINGE>) : go(chain_mma16_kernel<LOSS_SQUARED>);
+  if (b16) {
+    switch (c->loss) {
+      case WPSGD_LOSS_HINGE: return go(chain_mma16_kernel<LOSS_HINGE>);
+      case WPSGD_LOSS_LOGISTIC: return go(chain_mma16_kernel<LOSS_LOGISTIC>);
+      default: return go(chain_mma16_kernel<LOSS_SQUARED>);
+    }
+  }
   switch (c->loss) {
     case WPSGD_LOSS_HINGE: return go(chain_mma_kernel<LOSS_HINGE, 4>);
     case WPSGD_LOSS_LOGISTIC: return go(chain_mma_kernel<LOSS_LOGISTIC, 4>);

@@ -156,8 +156,6 @@ def test_large_d_falls_back_and_matches(P):
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
 @pytest.mark.parametrize("kind", ["block_fp32", "block_bf16", "warp", "mma8", "mma16"])
 def test_blocked_kernels_decaying_step_size(P, kind, loss):
-    if kind == "mma16" and loss == LOGISTIC:
-        pytest.skip("the 16-sample form has squared and hinge losses only")
     d = {"block_fp32": 1024, "block_bf16": 1000, "warp": 256, "mma8": 2048, "mma16": 2048}[kind]
     wl = wi.config2(k=4, d=d, m=96, base_steps=333)
     wl.n_steps[3] = 0
@@ -267,10 +265,7 @@ MMA_BLOCKS = [8, 16]
 
 
 def _mma(block, wl, **more):
-    """Options that select the tensor-core kernel with the given block size; the 16-sample form has no logistic loss."""
-    if block == 16 and wl.loss == LOGISTIC:
-        wl.loss = SQUARED
-        wl.y = (wl.y * 0.3).contiguous()
+    """Options that select the tensor-core kernel with the given block size."""
     return dict({"dense_variant": 8, "block_samples": block}, **more)
 
 
@@ -298,8 +293,6 @@ def test_mma_kernel_losses_and_widths(P, d, cluster, loss, block):
     if loss == SQUARED:
         wl.y = (wl.y * 0.3).contiguous()
     wl.X = wl.X.to(torch.bfloat16)
-    if block == 16 and loss == LOGISTIC:
-        pytest.skip("the 16-sample form has squared and hinge losses only")
     assert_parity(P, wl, _mma(block, wl, cluster=cluster))
 
 
@@ -351,11 +344,6 @@ def test_mma_kernel_limits(P, block):
     with pytest.raises(P.WpsgdError) as e:
         gpu_solve(P, wl, {"dense_variant": 8, "block_samples": block, "cluster": 16})
     assert e.value.status_name == "INVALID_ARG"
-    if block == 16:  # logistic loss: the 16-sample form is refused, the default falls back to 8 samples
-        with pytest.raises(P.WpsgdError) as e:
-            gpu_solve(P, wl, {"dense_variant": 8, "block_samples": 16})
-        assert e.value.status_name == "UNSUPPORTED"
-        assert_parity(P, wl, {"dense_variant": 8})
 
 
 @pytest.mark.parametrize("d,cluster", [(1024, 1), (4096, 2), (4096, 4)])
