@@ -85,11 +85,14 @@ wpsgd_status wpsgd_destroy(wpsgd_ctx* ctx);
  *                     one warp per node. 4: blocked form (8 samples per synchronisation), one CTA per node. 5: blocked
  *                     form, one warp per node (rows of at most 64 16-byte chunks). 8: blocked form for bf16 rows, Gram
  *                     block and margins from mma.sync tensor-core instructions, columns of a node split over a
- *                     thread-block cluster (what 0 picks for aligned bf16 rows of 2048 columns and more). The blocked
- *                     forms (4, 5, 8) take both step-size schedules and need eta0 * lambda <= 0.25.
+ *                     thread-block cluster (what 0 picks for aligned bf16 rows of 2048 columns and more). 9: blocked
+ *                     form (16 samples) for fp32 rows with a node's columns split over a cluster, at most 256 columns
+ *                     per CTA (what 0 picks for rows of 512 columns and more when the nodes are few enough for clusters
+ *                     of 4 or 8 on the GPU's SMs). The blocked forms (4, 5, 8, 9) take both step-size schedules and
+ *                     need eta0 * lambda <= 0.25.
  *   "sparse_variant"  kernel for CSR rows. 0 (default) and 2: blocks of up to 64 steps run in a shared-memory cache of
  *                     the model entries they touch. 1: one step per round trip to the model in global memory.
- *   "cluster"         CTAs per node of variant 8: 0 (default) chosen from d, else 1, 2, 4 or 8.
+ *   "cluster"         CTAs per node of variants 8 and 9: 0 (default) chosen from d (and the node count), else 1, 2, 4 or 8.
  *   "block_samples"   samples per block of variant 8: 0 (default) 16 when the rows fit, else 8; 8 or 16 to force one.
  *   "threads"         threads per node of variants 2 and 4, warps x 32 per CTA of variant 5; 0 (default): chosen from d.
  *   "prefetch"        rows in flight per chain of variants 2, 3 and of sparse variant 1; 0 (default): chosen.

@@ -434,12 +434,71 @@ bool mma_kernel_fits(const wpsgd_ctx* c, bool aligned, ClusterShape* out) {
   out->stages = stages;
   // 16 samples per block (squared and hinge losses): half as many hand-offs per sample; one CTA per SM
   int s16 = c->opt_stages > 0 ? std::min(c->opt_stages, 8) : 2;
-  while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16).total > kSmemBudget) --s16;
+  while (s16 >= 2 && Mma16Smem(s16, (size_t)cpc * 16, 2).total > kSmemBudget) --s16;
   out->stages16 = s16 >= 2 ? s16 : 0;
   const bool can16 = out->stages16 > 0;
   out->block = (c->opt_block_samples == 16 || (c->opt_block_samples == 0 && can16)) ? 16 : 8;
   if (out->block == 16 && !can16) return false;
   return true;
+}
+
+// ---- fp32 rows: the 16-sample cluster kernel with the Gram block on the fp32 pipes -------------------------------------
+// A chain is spread over as many CTAs as idle SMs allow (a cluster of 2, 4 or 8), each with at most 64 chunks of 4
+// columns: meant for few, wide chains that would otherwise hold one SM each.
+constexpr int kF16Stages = 3;
+bool f16_kernel_fits(const wpsgd_ctx* c, int nk, bool aligned, ClusterShape* out) {
+  if (!aligned || (double)c->eta0 * (double)c->lambda > 0.25) return false;
+  const long long chunks = c->d / 4;
+  int C = c->opt_cluster;
+  if (C <= 0) {
+    C = 8;
+    while (C > 1 && ((long long)nk * C > 148 || (chunks + C - 1) / C < 8)) C /= 2;
+  }
+  if (C != 1 && C != 2 && C != 4 && C != 8) return false;
+  const long long cpc = (chunks + C - 1) / C;
+  if (cpc < 1 || cpc > 64 || (long long)(C - 1) * cpc >= chunks) return false;
+  if (Mma16Smem(kF16Stages, (size_t)cpc * 16, 3).total > kSmemBudget) return false;
+  out->C = C;
+  out->cpc = (int)cpc;
+  out->math_warps = 8;
+  out->stages16 = kF16Stages;
+  out->block = 16;
+  return true;
+}
+
+wpsgd_status launch_f16(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
+  ClusterParams cp;
+  cp.b.c = p;
+  cp.b.stages = sh.stages16;
+  cp.b.eta_lambda = (double)c->eta0 * (double)c->lambda;
+  cp.b.spin_limit = c->opt_spin_limit;
+  cp.b.drop_block = c->opt_drop_block;
+  cp.b.group_order = nullptr;
+  cp.chunks_per_cta = sh.cpc;
+  const size_t smem = Mma16Smem(sh.stages16, (size_t)sh.cpc * 16, 3).total;
+  auto go = [&](auto kern) -> wpsgd_status {
+    CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.k * sh.C));
+    cfg.blockDim = dim3((unsigned)(64 + 32 * sh.math_warps));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)sh.C;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    CU_TRY(c, cudaLaunchKernelEx(&cfg, kern, cp));
+    c->launches++;
+    return WPSGD_OK;
+  };
+  switch (c->loss) {
+    case WPSGD_LOSS_HINGE: return go(chain_mma16_kernel<LOSS_HINGE, float>);
+    case WPSGD_LOSS_LOGISTIC: return go(chain_mma16_kernel<LOSS_LOGISTIC, float>);
+    default: return go(chain_mma16_kernel<LOSS_SQUARED, float>);
+  }
 }
 
 wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& sh) {
@@ -453,7 +512,7 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   cp.chunks_per_cta = sh.cpc;
   const bool b16 = sh.block == 16;
   if (b16) cp.b.stages = sh.stages16;
-  const size_t smem = b16 ? Mma16Smem(sh.stages16, (size_t)sh.cpc * 16).total : MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
+  const size_t smem = b16 ? Mma16Smem(sh.stages16, (size_t)sh.cpc * 16, 2).total : MmaSmem(sh.stages, (size_t)sh.cpc * 16, MMA_SLOTS).total;
   auto go = [&](auto kern) -> wpsgd_status {
     CU_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
@@ -474,9 +533,9 @@ wpsgd_status launch_mma(wpsgd_ctx* c, const ChainParams& p, const ClusterShape& 
   };
   if (b16) {
     switch (c->loss) {
-      case WPSGD_LOSS_HINGE: return go(chain_mma16_kernel<LOSS_HINGE>);
-      case WPSGD_LOSS_LOGISTIC: return go(chain_mma16_kernel<LOSS_LOGISTIC>);
-      default: return go(chain_mma16_kernel<LOSS_SQUARED>);
+      case WPSGD_LOSS_HINGE: return go(chain_mma16_kernel<LOSS_HINGE, __nv_bfloat16>);
+      case WPSGD_LOSS_LOGISTIC: return go(chain_mma16_kernel<LOSS_LOGISTIC, __nv_bfloat16>);
+      default: return go(chain_mma16_kernel<LOSS_SQUARED, __nv_bfloat16>);
     }
   }
   switch (c->loss) {
@@ -602,10 +661,12 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
   const bool block_ok = block_kernel_fits<XT>(c, aligned, &bthreads, &bR, &bstages);
   int wR = 0, wstages = 0, wwarps = 0;
   const bool block_warp_ok = block_warp_kernel_fits<XT>(c, p.k, aligned, &wR, &wstages, &wwarps);
-  ClusterShape mma_shape;
+  ClusterShape mma_shape, f16_shape;
   const bool mma_ok = sizeof(XT) == 2 && mma_kernel_fits(c, aligned, &mma_shape);
+  const bool f16_ok = sizeof(XT) == 4 && f16_kernel_fits(c, p.k, aligned, &f16_shape);
   if (variant == 0) {
     if (!aligned) variant = 1;
+    else if (f16_ok && f16_shape.C >= 4 && chunks >= 128) variant = 9;  // few wide fp32 chains: spread each over idle SMs
     else if (chunks <= 64) variant = block_warp_ok ? 5 : 3;
     else if (sizeof(XT) == 2 && chunks >= 256 && mma_ok) variant = 8;  // wide bf16 rows: tensor-core cluster kernel
     else if (block_ok) variant = 4;
@@ -625,6 +686,13 @@ wpsgd_status launch_dense(wpsgd_ctx* c, const ChainParams& p) {
                   "tensor-core cluster kernel needs bf16 rows, 16-byte aligned, eta*lambda <= 0.25, a "
                   "cluster of 1, 2, 4 or 8 CTAs with at most 256 chunks of a row each and at most 16 math warps in all");
     return launch_mma(c, p, sh);
+  }
+  if (variant == 9) {
+    if (!f16_ok)
+      return fail(c, WPSGD_ERR_UNSUPPORTED,
+                  "16-sample cluster kernel for fp32 rows needs 16-byte aligned rows, eta*lambda <= 0.25 and a cluster of "
+                  "1, 2, 4 or 8 CTAs with at most 64 chunks of a row each");
+    return launch_f16(c, p, f16_shape);
   }
   if (variant == 4) {
     if (!block_ok)
@@ -896,7 +964,7 @@ wpsgd_status wpsgd_set_option(wpsgd_ctx* c, const char* name, int64_t value) {
   if (!c || !name) return fail(c, WPSGD_ERR_INVALID_ARG, "ctx or name is NULL");
   const std::string n(name);
   if (n == "dense_variant") {
-    if (value < 0 || value > 8 || value == 6 || value == 7) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..5 or 8");
+    if (value < 0 || value > 9 || value == 6 || value == 7) return fail(c, WPSGD_ERR_INVALID_ARG, "dense_variant must be 0..5, 8 or 9");
     c->opt_variant = (int)value;
   } else if (n == "prefetch") {
     if (value < 0 || value > 64) return fail(c, WPSGD_ERR_INVALID_ARG, "prefetch must be 0..64");

@@ -154,20 +154,21 @@ def test_large_d_falls_back_and_matches(P):
 
 # ---- blocked kernels with the decaying step size eta0 / sqrt(n): per-block tables instead of powers of one factor -------
 @pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
-@pytest.mark.parametrize("kind", ["block_fp32", "block_bf16", "warp", "mma8", "mma16"])
+@pytest.mark.parametrize("kind", ["block_fp32", "block_bf16", "warp", "mma8", "mma16", "f32x16"])
 def test_blocked_kernels_decaying_step_size(P, kind, loss):
-    d = {"block_fp32": 1024, "block_bf16": 1000, "warp": 256, "mma8": 2048, "mma16": 2048}[kind]
+    d = {"block_fp32": 1024, "block_bf16": 1000, "warp": 256, "mma8": 2048, "mma16": 2048, "f32x16": 1024}[kind]
     wl = wi.config2(k=4, d=d, m=96, base_steps=333)
     wl.n_steps[3] = 0
     wl.loss, wl.sched, wl.eta0, wl.lam = loss, 1, 0.3, 0.05  # eta_n lambda from 1.5e-2 down: the factors differ step by step
     if loss == SQUARED:
         wl.y = (wl.y * 0.3).contiguous()
     wl.w0 = torch.full((d,), 0.05)
-    if kind != "block_fp32" and kind != "warp":
+    if kind not in ("block_fp32", "warp", "f32x16"):
         wl.X = wl.X.to(torch.bfloat16)
     opts = {"block_fp32": {"dense_variant": 4}, "block_bf16": {"dense_variant": 4}, "warp": {"dense_variant": 5},
             "mma8": {"dense_variant": 8, "block_samples": 8, "cluster": 2},
-            "mma16": {"dense_variant": 8, "block_samples": 16, "cluster": 2}}[kind]
+            "mma16": {"dense_variant": 8, "block_samples": 16, "cluster": 2},
+            "f32x16": {"dense_variant": 9, "cluster": 4}}[kind]
     assert_parity(P, wl, opts)
 
 
@@ -373,8 +374,78 @@ def test_mma_kernel_bounded_waits_report_timeout_and_context_survives(P, d, clus
     assert rel_l2(v, ov) <= 1e-4
 
 
+# ---- fp32 rows, 16 samples per block, a chain spread over a cluster (Gram block on the fp32 pipes) ----------------------
+@pytest.mark.parametrize("d,cluster", [(1024, 8), (1024, 4), (512, 2), (256, 1), (1000, 8), (36, 1), (2048, 8)])
+@pytest.mark.parametrize("loss", [HINGE, LOGISTIC, SQUARED])
+def test_f32_cluster_kernel_losses_and_widths(P, d, cluster, loss):
+    wl = wi.config2(k=3, d=d, m=48, base_steps=210)
+    wl.loss = loss
+    if loss == SQUARED:
+        wl.y = (wl.y * 0.3).contiguous()
+    assert_parity(P, wl, {"dense_variant": 9, "cluster": cluster})
+
+
+@pytest.mark.parametrize("n_steps", [(1, 7, 8), (9, 15, 16), (17, 0, 64), (333, 250, 3), (31, 32, 33)])
+@pytest.mark.parametrize("cluster", [1, 4])
+def test_f32_cluster_kernel_block_boundaries_and_empty_chains(P, n_steps, cluster):
+    wl = wi.config2(k=3, d=256, m=64, base_steps=8)
+    wl.n_steps = np.array(n_steps, dtype=np.int64)
+    wl.w0 = torch.full((256,), 0.1)
+    assert_parity(P, wl, {"dense_variant": 9, "cluster": cluster})
+
+
+def test_f32_cluster_kernel_default_shape_and_continue(P):
+    wl_cpu = wi.config2(k=5, d=1024, m=96, base_steps=700)
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("dense_variant", 9)
+        first = np.minimum(wl.n_steps, 301)
+        ctx.run(wl.X, wl.y, wl.shard_off, first, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+        ctx.continue_(wl.X, wl.y, wl.shard_off, wl.n_steps - first)
+        seg = ctx.get_models().cpu().numpy()
+        ctx.check()
+    oW = oracle.run_dense(wl_cpu.X, wl_cpu.y, wl.shard_off, wl.n_steps, wl.d, wl.eta0, wl.sched, wl.lam, wl.loss, wl.seed)
+    for j in range(wl.k):
+        assert rel_l2(seg[j], oW[j]) <= 1e-4
+
+
+def test_f32_cluster_kernel_limits(P):
+    wl = wi.config2(k=2, d=2048, m=16, base_steps=20)  # 512 chunks: one CTA would hold more than 64
+    with pytest.raises(P.WpsgdError) as e:
+        gpu_solve(P, wl, {"dense_variant": 9, "cluster": 4})
+    assert e.value.status_name == "UNSUPPORTED"
+    wl.X = wl.X.to(torch.bfloat16)
+    with pytest.raises(P.WpsgdError) as e:
+        gpu_solve(P, wl, {"dense_variant": 9})
+    assert e.value.status_name == "UNSUPPORTED"
+
+
+@pytest.mark.parametrize("d,cluster", [(256, 1), (1024, 4), (1024, 8)])
+def test_f32_cluster_kernel_bounded_waits_report_timeout_and_context_survives(P, d, cluster):
+    # the rows of block 3 are never requested (test hook): the bounded wait for them runs out, every CTA of the
+    # cluster is told, all leave in step, and the next run is clean
+    wl_cpu = wi.config2(k=3, d=d, m=32, base_steps=120)
+    wl = wl_cpu.to("cuda")
+    with P.Context(wl.k, wl.d) as ctx:
+        ctx.set_option("dense_variant", 9)
+        ctx.set_option("cluster", cluster)
+        ctx.set_option("spin_limit", 2000)
+        ctx.set_option("test_drop_block", 3)
+        ctx.run_workload(wl)
+        with pytest.raises(P.WpsgdError) as e:
+            ctx.check()
+        assert e.value.status_name == "TIMEOUT"
+        ctx.set_option("test_drop_block", -1)
+        ctx.set_option("spin_limit", 1 << 20)
+        ctx.run_workload(wl)
+        v = ctx.combine().cpu().numpy()
+        ctx.check()
+    ov, _, _ = oracle.solve(wl_cpu)
+    assert rel_l2(v, ov) <= 1e-4
+
+
 # ---- logistic loss: blocks whose steps move the margins far take the direct evaluation ---------------------------------
-@pytest.mark.parametrize("variant,d", [(4, 1024), (5, 128), (8, 1024)])
+@pytest.mark.parametrize("variant,d", [(4, 1024), (5, 128), (8, 1024), (9, 1024)])
 def test_logistic_large_steps_between_correlated_rows(P, variant, d):
     # rows that are nearly parallel (large Gram entries) and a large step size: inside a block of 8 samples the
     # margins move by much more than the range of the cubic expansion of the logistic factor
@@ -388,11 +459,13 @@ def test_logistic_large_steps_between_correlated_rows(P, variant, d):
     assert_parity(P, wl, {"dense_variant": variant})
 
 
-def test_blocked_kernel_is_the_default_for_large_aligned_d(P):
-    wl = wi.config2(k=4, d=1024, m=64, base_steps=100).to("cuda")
+@pytest.mark.parametrize("k,variant", [(4, 9), (40, 4)])
+def test_default_kernels_for_large_aligned_fp32_rows(P, k, variant):
+    # few chains: each spread over a cluster of idle SMs (16 samples per block); many chains: one CTA each (8 per block)
+    wl = wi.config2(k=k, d=1024, m=64, base_steps=100).to("cuda")
     with P.Context(wl.k, wl.d) as a, P.Context(wl.k, wl.d) as b:
         a.run_workload(wl)
-        b.set_option("dense_variant", 4)
+        b.set_option("dense_variant", variant)
         b.run_workload(wl)
         np.testing.assert_array_equal(a.get_models().cpu().numpy(), b.get_models().cpu().numpy())
         a.check()
