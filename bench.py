@@ -45,10 +45,11 @@ N_SMS = 148
 # DRAM bytes (read + write) per launch of the chain kernel from an ncu capture, with the hash of the
 # kernel sources the capture was taken from; reported as null once the sources have changed.
 NCU_TRAFFIC = {
-    "config3": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 26347168248,
+    "config3": {"src_sha": "5464430f1e53acb2", "bytes_per_launch": 26347713776,
                 "note": "captured with 2048 rows per node (2 GiB on the device): same step counts and kernel work per launch, no scaling"},
-    "config5": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 15944920632, "note": "full-size capture"},
-    "config4": {"src_sha": "9c395b1487fcc28d", "bytes_per_launch": 4306268816, "note": "full-size capture"},
+    "config5": {"src_sha": "5464430f1e53acb2", "bytes_per_launch": 15943503448, "note": "full-size capture"},
+    "config4": {"src_sha": "5464430f1e53acb2", "bytes_per_launch": 4299267560, "note": "full-size capture"},
+    "config2": {"src_sha": "5464430f1e53acb2", "bytes_per_launch": 604431360, "note": "full-size capture"},
 }
 
 
@@ -127,6 +128,12 @@ def ctas_of(wl) -> int:
     if wl.sparse:
         return wl.k
     chunks = wl.d // (8 if wl.xtype == 1 else 4)
+    if wl.xtype != 1 and chunks >= 128:   # few wide fp32 chains: a cluster of 4 or 8 CTAs per node when the SMs allow
+        c = 8
+        while c > 1 and (wl.k * c > N_SMS or (chunks + c - 1) // c < 8):
+            c //= 2
+        if c >= 4 and (chunks + c - 1) // c <= 64:
+            return wl.k * c
     if chunks <= 64:
         return (wl.k + 3) // 4            # four nodes (warps) per CTA
     if wl.xtype == 1 and chunks >= 256:
