@@ -179,9 +179,13 @@ def config4(k=64, d=1 << 20, m=65536, base_steps=65536, mean_nnz=40.0, max_nnz=1
     perm = torch.randperm(d, generator=g, device=device)  # rank -> column (hot columns scattered)
     # sparse w*: ceil(0.01 d) nonzeros on columns drawn from the same law
     n_star = max(1, math.ceil(0.01 * d))
-    w_star = torch.zeros(d, dtype=torch.float32, device=device)
     star_cols = perm[_zipf_draw(cdf, (n_star,), g)]
-    w_star[star_cols] = torch.randn(n_star, generator=g, device=device)
+    star_vals = torch.randn(n_star, generator=g, device=device)
+    # the hot columns are drawn more than once: the last draw of a column stands (written out on the host, in order,
+    # because a device scatter with repeated indices keeps whichever write lands last)
+    w_host = np.zeros(d, dtype=np.float32)
+    w_host[star_cols.cpu().numpy()] = star_vals.cpu().numpy()
+    w_star = torch.from_numpy(w_host).to(device)
 
     N = k * m
     nnz_all, cols_all, y_all = [], [], []
